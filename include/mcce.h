@@ -1,0 +1,163 @@
+/*
+ * mcce -- cache-conditional MoE decode step for many independent token streams (NVIDIA B200, sm_100a).
+ *
+ * C ABI of libmcce.so.  Plain pointers and sizes only; every pointer is marked HOST or DEVICE.
+ * The method is "Mixture of Cache-Conditional Experts" (arXiv 2412.00099); the citations below name
+ * the equation, section or algorithm of that paper which defines each operation.
+ *
+ * Notation (paper, Sec. 2.1 / 2.2 / 3.3): N = E routed experts per layer, top-K selection, top-J
+ * guaranteed experts, cache set C of `cache_capacity` experts per (stream, layer), promotion strength
+ * lambda, logit range Delta_avg.  S independent token streams, L MoE layers, hidden size d, expert
+ * intermediate size I.  Streams and layers are independent of one another; tokens of one stream are
+ * sequential because the cache state carries over.
+ *
+ * Ownership: the caller owns every buffer, including the workspace, and keeps them alive until
+ * mcce_destroy.  The library allocates no device memory and creates no streams.  Weights are borrowed.
+ * Errors: every call returns 0 on success or a negative MCCE_E* code; nothing throws, aborts or prints.
+ * Kernel launches are asynchronous on the given stream unless a function says that it synchronises.
+ * A context is not thread-safe; distinct contexts are independent.
+ */
+#ifndef MCCE_H_
+#define MCCE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  MCCE_OK = 0,
+  MCCE_EINVAL = -1,   /* bad argument or unsupported configuration                      */
+  MCCE_ENOSPC = -2,   /* workspace too small                                            */
+  MCCE_ESTATE = -3,   /* weights not set, or a counter would overflow (reset needed)    */
+  MCCE_ECUDA = -4,    /* a CUDA call failed; see mcce_last_cuda_error                   */
+  MCCE_ETIMEOUT = -5  /* a bounded wait inside a kernel gave up; the context stays usable */
+};
+
+enum { MCCE_F32 = 0, MCCE_BF16 = 1 };
+enum { MCCE_DELTA_RUNNING = 0, MCCE_DELTA_FIXED = 1 };
+enum { MCCE_FFN_AUTO = 0, MCCE_FFN_SIMT = 1, MCCE_FFN_TENSOR = 2 };
+
+typedef struct mcce_ctx mcce_ctx; /* opaque; host memory owned by the library */
+
+typedef struct {
+  int32_t n_layers;       /* L >= 1                                                              */
+  int32_t n_experts;      /* E = N routed experts per layer, 1..256                              */
+  int32_t top_k;          /* K, 1..min(E,16)                                                     */
+  int32_t top_j;          /* J, 0..K: router's top-J experts are always selected (Sec. 3.3)      */
+  int32_t n_shared;       /* always-on experts per layer, weight 1, never cached, >= 0           */
+  int32_t d_model;        /* d, multiple of 8                                                    */
+  int32_t d_ff;           /* I, multiple of 8                                                    */
+  int32_t cache_capacity; /* C >= 1 experts per (stream, layer); C >= E means nothing is evicted */
+  int32_t n_streams;      /* S >= 1                                                              */
+  float lambda;           /* promotion strength of Eq. 7, finite, >= 0 (paper: [0,1])            */
+  int32_t delta_mode;     /* MCCE_DELTA_RUNNING: Delta_avg is the cumulative mean, per (stream,
+                             layer), of max(z)-min(z) including the current token (Eq. 8);
+                             MCCE_DELTA_FIXED: per-layer constants given to mcce_set_router
+                             (appendix "Logit Range Estimation")                                 */
+  int32_t renorm;         /* 1: weights renormalised over the K selected experts (Sec. 2.1)      */
+  int32_t hidden_dtype;   /* MCCE_F32 or MCCE_BF16                                               */
+  int32_t weight_dtype;   /* expert weights; must equal hidden_dtype                             */
+  int32_t ffn_impl;       /* MCCE_FFN_AUTO picks the tensor-core path when it applies            */
+  int32_t device;         /* CUDA device ordinal                                                 */
+} mcce_config;
+
+typedef struct {
+  int64_t steps;       /* (stream, token, layer) routing steps                                   */
+  int64_t selections;  /* K * steps, denominator of Eq. 4                                        */
+  int64_t misses;      /* selected experts absent from the cache as it was before the token      */
+  int64_t cold_misses; /* misses on experts that had never been resident (compulsory misses)     */
+} mcce_stats;
+
+/* Bytes of DEVICE workspace mcce_create needs for this configuration (0 if the config is invalid). */
+size_t mcce_workspace_bytes(const mcce_config* cfg /*HOST*/);
+
+/* Validates cfg, carves `workspace` (DEVICE, 256-byte aligned, >= mcce_workspace_bytes) into the
+ * state arrays, zeroes them (cache empty) and returns a context.  Synchronises the device. */
+int mcce_create(const mcce_config* cfg /*HOST*/, void* workspace /*DEVICE*/, size_t workspace_bytes,
+                mcce_ctx** out /*HOST*/);
+int mcce_destroy(mcce_ctx* ctx);
+
+/* Router G of Eq. 3: z = W_r[l] x.  Wr: DEVICE fp32 [L,E,d], row-major.  fixed_delta: DEVICE fp32 [L],
+ * required iff delta_mode == MCCE_DELTA_FIXED, else may be NULL.  Borrowed. */
+int mcce_set_router(mcce_ctx* ctx, const float* Wr, const float* fixed_delta);
+
+/* Experts E_i of Eq. 1 as SwiGLU: E_i(x) = W_d (silu(W_g x) * (W_u x)).  DEVICE, weight_dtype,
+ * row-major: Wg, Wu [L,E,I,d]; Wd [L,E,d,I]; shared experts shWg, shWu [L,n_shared,I,d],
+ * shWd [L,n_shared,d,I] (NULL when n_shared == 0).  Borrowed. */
+int mcce_set_experts(mcce_ctx* ctx, const void* Wg, const void* Wu, const void* Wd, const void* shWg,
+                     const void* shWu, const void* shWd);
+
+/* Empties every cache, or loads an initial cache content (Sec. 4.8 "Impact of Initial Cache State"):
+ * init_order HOST int32 [L,S,C], resident experts most-recently-used first, -1 padding; NULL = empty.
+ * These entries count as older than anything touched later.  Counters are zeroed.  The running
+ * Delta statistics are kept iff keep_delta_stats != 0, or replaced when delta_sum (HOST fp32 [L,S])
+ * is given together with delta_count (tokens it was summed over).  Synchronises. */
+int mcce_reset(mcce_ctx* ctx, const int32_t* init_order, int keep_delta_stats, const float* delta_sum,
+               int64_t delta_count);
+
+/* n_steps tokens of routing for every (stream, layer): Eq. 3 logits (or given logits), Eq. 8 range
+ * statistic, mask m~_t = cache OR top-J, Eq. 7 promotion z' = z + lambda*Delta_avg*m~_t, top-K of z'
+ * (ties to the lower expert index), weights = softmax of the UNMODIFIED z over the selected experts
+ * (Sec. 3.3), Eq. 4 miss counting against the cache as it was before the token, LRU update in which
+ * the selected expert with the higher router weight counts as older (Sec. 4.2).
+ *   hidden     DEVICE hidden_dtype [n_steps,L,S,d], or NULL
+ *   logits_in  DEVICE fp32 [n_steps,L,S,E], or NULL; exactly one of the two is non-NULL
+ *   sel_idx    DEVICE int32 [n_steps,L,S,K] out, rank order of z'
+ *   sel_w      DEVICE fp32  [n_steps,L,S,K] out
+ *   logits_out DEVICE fp32  [n_steps,L,S,E] out, optional: the logits the decision was taken on
+ */
+int mcce_route_step(mcce_ctx* ctx, int32_t n_steps, const void* hidden, const float* logits_in,
+                    int32_t* sel_idx, float* sel_w, float* logits_out, void* cuda_stream);
+
+/* Eq. 1 for one token of every (stream, layer): groups the (stream, slot) pairs by expert, runs the
+ * SwiGLU experts group by group and combines y = sum_k w_k E_sel_k(x) (slot order) + shared experts.
+ *   hidden DEVICE hidden_dtype [L,S,d]; sel_idx DEVICE int32 [L,S,K]; sel_w DEVICE fp32 [L,S,K];
+ *   y DEVICE fp32 [L,S,d] out.
+ * With bf16 weights the intermediate silu(g)*u is rounded to bf16 before the down projection. */
+int mcce_moe_forward(mcce_ctx* ctx, const void* hidden, const int32_t* sel_idx, const float* sel_w,
+                     float* y, void* cuda_stream);
+
+/* One whole decode step from HOST buffers: copies hidden [L,S,d] to the device, routes, runs the
+ * experts and copies y [L,S,d] (and, if non-NULL, sel_idx [L,S,K]) back.  Staging lives in the
+ * workspace.  hidden_host / y_host should be pinned.  Synchronises the stream before returning. */
+int mcce_decode_step_host(mcce_ctx* ctx, const void* hidden_host, float* y_host, int32_t* sel_idx_host,
+                          void* cuda_stream);
+
+/* Eq. 4 counters, summed over streams: total and per layer (HOST [L], may be NULL).  Synchronises.
+ * Also reports MCCE_ETIMEOUT if any kernel of this context gave up on a bounded wait. */
+int mcce_cache_stats(mcce_ctx* ctx, mcce_stats* total /*HOST*/, mcce_stats* per_layer /*HOST*/);
+
+/* Canonical cache state: order HOST int32 [L,S,C] most-recently-used first, -1 padded; optional
+ * ever HOST uint8 [L,S,E]; delta_sum HOST fp32 [L,S] and *delta_count (optional).  Synchronises. */
+int mcce_get_cache_state(mcce_ctx* ctx, int32_t* order, uint8_t* ever, float* delta_sum,
+                         int64_t* delta_count);
+
+/* Result of the expert-grouping pass of the last mcce_moe_forward (histogram, scan, stable scatter):
+ * offsets HOST int32 [L,E+1]; perm HOST int32 [L,S*K], perm[l][pos] = s*K+slot of the pair placed at
+ * pos, pairs of one expert contiguous and in increasing (s,slot) order.  Synchronises. */
+int mcce_get_grouping(mcce_ctx* ctx, int32_t* offsets, int32_t* perm);
+
+/* Seeded synthetic inputs (counter-based: Philox4x32-10 keyed by (seed, 0), counter = (element
+ * block, t, tensor_id), Box-Muller with fixed-order fp32 series); no counterpart in the paper, whose
+ * inputs are text corpora.  out DEVICE, dtype MCCE_F32/MCCE_BF16; elements [start, start+count) of the
+ * tensor, value = std * n.  start must be a multiple of 4. */
+int mcce_gen_normal(void* out, int32_t dtype, uint64_t start, uint64_t count, uint32_t seed,
+                    uint32_t tensor_id, uint32_t t, float std, void* cuda_stream);
+/* AR(1) hidden states: h <- (t==0 ? n_t : rho*h + c*n_t) on state DEVICE fp32 [count]; emits
+ * x = h + offset_scale * n_offset (offset omitted when offset_scale == 0) as dtype.  count % 4 == 0. */
+int mcce_gen_hidden_step(float* state, void* x_out, int32_t dtype, uint64_t count, uint32_t seed,
+                         uint32_t t, float rho, float c, float offset_scale, void* cuda_stream);
+/* Raw Philox words, DEVICE uint32 [n_blocks,4], for checking the generator bit by bit. */
+int mcce_gen_philox_words(uint32_t* out, uint64_t start_block, uint64_t n_blocks, uint32_t seed,
+                          uint32_t tensor_id, uint32_t t, void* cuda_stream);
+
+const char* mcce_strerror(int code);
+int mcce_last_cuda_error(const mcce_ctx* ctx); /* cudaError_t of the last failed CUDA call */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MCCE_H_ */

@@ -1,0 +1,366 @@
+// Host side of libmcce.so: configuration checks, workspace layout, and the entry points of mcce.h.
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "common.cuh"
+#include "ffn_tc.cuh"
+
+using namespace mcce;
+
+struct mcce_ctx {
+  mcce_config cfg;
+  int EW;
+  size_t rows;  // rows of H / O: L*S*K routed pairs + L*n_sh*S shared
+  // workspace pieces (device)
+  uint32_t *stamp, *ever, *miss, *cold, *err;
+  float* sum_range;
+  unsigned long long* stats_dev;
+  int32_t *offsets, *perm, *inv;
+  void *Xg, *H;
+  float* O;
+  void* stage_hidden;
+  int32_t* stage_sel;
+  float *stage_w, *stage_y;
+  // borrowed weights
+  const float *Wr, *fixed_delta;
+  const void *Wg, *Wu, *Wd, *shWg, *shWu, *shWd;
+  // host-side counters
+  uint64_t tok, delta_cnt, steps_since_reset;
+  int last_cuda;
+  int use_tc;
+  TcPlan tc;
+};
+
+namespace {
+
+constexpr size_t kAlign = 256;
+size_t up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+bool valid(const mcce_config* c) {
+  if (!c) return false;
+  if (c->n_layers < 1 || c->n_streams < 1) return false;
+  if (c->n_experts < 1 || c->n_experts > kMaxE) return false;
+  if (c->top_k < 1 || c->top_k > kMaxK || c->top_k > c->n_experts) return false;
+  if (c->top_j < 0 || c->top_j > c->top_k) return false;
+  if (c->n_shared < 0 || c->cache_capacity < 1) return false;
+  if (c->d_model < 8 || c->d_model % 8 || c->d_ff < 8 || c->d_ff % 8) return false;
+  if (!(c->lambda >= 0.f) || !isfinite(c->lambda)) return false;
+  if (c->delta_mode != MCCE_DELTA_RUNNING && c->delta_mode != MCCE_DELTA_FIXED) return false;
+  if (c->hidden_dtype != MCCE_F32 && c->hidden_dtype != MCCE_BF16) return false;
+  if (c->weight_dtype != c->hidden_dtype) return false;
+  if (c->ffn_impl < MCCE_FFN_AUTO || c->ffn_impl > MCCE_FFN_TENSOR) return false;
+  if (c->ffn_impl == MCCE_FFN_TENSOR && !tc_applicable(*c)) return false;
+  if (c->device < 0) return false;
+  return true;
+}
+
+struct Layout {
+  size_t stamp, ever, sum_range, miss, cold, err, stats, offsets, perm, inv, Xg, H, O, st_hidden, st_sel, st_w, st_y,
+      total;
+};
+
+Layout layout_of(const mcce_config& c) {
+  const size_t L = c.n_layers, S = c.n_streams, E = c.n_experts, K = c.top_k, d = c.d_model, I = c.d_ff;
+  const size_t EW = (E + 31) / 32, esz = c.hidden_dtype == MCCE_BF16 ? 2 : 4;
+  const size_t rows = L * S * K + L * (size_t)c.n_shared * S;
+  Layout o;
+  size_t p = 0;
+  auto take = [&](size_t bytes) {
+    const size_t at = p;
+    p += up(bytes);
+    return at;
+  };
+  o.stamp = take(L * S * E * 4);
+  o.ever = take(L * S * EW * 4);
+  o.sum_range = take(L * S * 4);
+  o.miss = take(L * S * 4);
+  o.cold = take(L * S * 4);
+  o.err = take(64);
+  o.stats = take(L * 2 * 8);
+  o.offsets = take(L * (E + 1) * 4);
+  o.perm = take(L * S * K * 4);
+  o.inv = take(L * S * K * 4);
+  o.Xg = take((L * S * K + 256) * d * esz);  // slack rows: tensor-core tiles read past a group's end
+  o.H = take((rows + 256) * I * esz);
+  o.O = take(rows * d * 4);
+  o.st_hidden = take(L * S * d * esz);
+  o.st_sel = take(L * S * K * 4);
+  o.st_w = take(L * S * K * 4);
+  o.st_y = take(L * S * d * 4);
+  o.total = p;
+  return o;
+}
+
+int cuda_fail(mcce_ctx* ctx, cudaError_t e) {
+  if (ctx) ctx->last_cuda = (int)e;
+  return MCCE_ECUDA;
+}
+#define CK(call)                                      \
+  do {                                                \
+    cudaError_t e_ = (call);                          \
+    if (e_ != cudaSuccess) return cuda_fail(ctx, e_); \
+  } while (0)
+
+FfnParams ffn_params(const mcce_ctx* ctx, const void* hidden, const float* sel_w, float* y) {
+  const mcce_config& c = ctx->cfg;
+  FfnParams f;
+  f.L = c.n_layers, f.S = c.n_streams, f.E = c.n_experts, f.K = c.top_k, f.n_sh = c.n_shared;
+  f.d = c.d_model, f.I = c.d_ff, f.bf16 = c.hidden_dtype == MCCE_BF16;
+  f.hidden = hidden;
+  f.Wg = ctx->Wg, f.Wu = ctx->Wu, f.Wd = ctx->Wd, f.shWg = ctx->shWg, f.shWu = ctx->shWu, f.shWd = ctx->shWd;
+  f.offsets = ctx->offsets, f.perm = ctx->perm, f.inv = ctx->inv, f.sel_w = sel_w;
+  f.Xg = ctx->Xg, f.H = ctx->H, f.O = ctx->O, f.y = y;
+  return f;
+}
+
+}  // namespace
+
+extern "C" size_t mcce_workspace_bytes(const mcce_config* cfg) { return valid(cfg) ? layout_of(*cfg).total : 0; }
+
+extern "C" int mcce_create(const mcce_config* cfg, void* workspace, size_t workspace_bytes, mcce_ctx** out) {
+  if (!out) return MCCE_EINVAL;
+  *out = nullptr;
+  if (!valid(cfg) || !workspace || ((uintptr_t)workspace % kAlign)) return MCCE_EINVAL;
+  const Layout lo = layout_of(*cfg);
+  if (workspace_bytes < lo.total) return MCCE_ENOSPC;
+  mcce_ctx* ctx = new (std::nothrow) mcce_ctx();
+  if (!ctx) return MCCE_EINVAL;
+  memset(ctx, 0, sizeof(*ctx));
+  ctx->cfg = *cfg;
+  ctx->EW = (cfg->n_experts + 31) / 32;
+  ctx->rows = (size_t)cfg->n_layers * cfg->n_streams * cfg->top_k + (size_t)cfg->n_layers * cfg->n_shared * cfg->n_streams;
+  char* w = (char*)workspace;
+  ctx->stamp = (uint32_t*)(w + lo.stamp), ctx->ever = (uint32_t*)(w + lo.ever);
+  ctx->sum_range = (float*)(w + lo.sum_range);
+  ctx->miss = (uint32_t*)(w + lo.miss), ctx->cold = (uint32_t*)(w + lo.cold), ctx->err = (uint32_t*)(w + lo.err);
+  ctx->stats_dev = (unsigned long long*)(w + lo.stats);
+  ctx->offsets = (int32_t*)(w + lo.offsets), ctx->perm = (int32_t*)(w + lo.perm), ctx->inv = (int32_t*)(w + lo.inv);
+  ctx->Xg = w + lo.Xg, ctx->H = w + lo.H, ctx->O = (float*)(w + lo.O);
+  ctx->stage_hidden = w + lo.st_hidden, ctx->stage_sel = (int32_t*)(w + lo.st_sel);
+  ctx->stage_w = (float*)(w + lo.st_w), ctx->stage_y = (float*)(w + lo.st_y);
+  ctx->use_tc = cfg->ffn_impl != MCCE_FFN_SIMT && tc_applicable(*cfg);
+  cudaError_t e = cudaSetDevice(cfg->device);
+  // state arrays and the activation buffers start at zero (the slack rows must hold finite values)
+  if (e == cudaSuccess) e = cudaMemset(w, 0, lo.O);
+  if (e == cudaSuccess) e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) {
+    delete ctx;
+    return MCCE_ECUDA;
+  }
+  *out = ctx;
+  return MCCE_OK;
+}
+
+extern "C" int mcce_destroy(mcce_ctx* ctx) {
+  if (!ctx) return MCCE_EINVAL;
+  delete ctx;
+  return MCCE_OK;
+}
+
+extern "C" int mcce_set_router(mcce_ctx* ctx, const float* Wr, const float* fixed_delta) {
+  if (!ctx || !Wr) return MCCE_EINVAL;
+  if (ctx->cfg.delta_mode == MCCE_DELTA_FIXED && !fixed_delta) return MCCE_EINVAL;
+  if ((uintptr_t)Wr % 16) return MCCE_EINVAL;
+  ctx->Wr = Wr;
+  ctx->fixed_delta = fixed_delta;
+  return MCCE_OK;
+}
+
+extern "C" int mcce_set_experts(mcce_ctx* ctx, const void* Wg, const void* Wu, const void* Wd, const void* shWg,
+                                const void* shWu, const void* shWd) {
+  if (!ctx || !Wg || !Wu || !Wd) return MCCE_EINVAL;
+  if (ctx->cfg.n_shared > 0 && (!shWg || !shWu || !shWd)) return MCCE_EINVAL;
+  const void* all[6] = {Wg, Wu, Wd, shWg, shWu, shWd};
+  for (const void* q : all)
+    if ((uintptr_t)q % 16) return MCCE_EINVAL;
+  ctx->Wg = Wg, ctx->Wu = Wu, ctx->Wd = Wd, ctx->shWg = shWg, ctx->shWu = shWu, ctx->shWd = shWd;
+  if (ctx->use_tc) {
+    const int rc = tc_plan(ctx->cfg, Wg, Wu, Wd, shWg, shWu, shWd, ctx->Xg, ctx->H, &ctx->tc);
+    if (rc != MCCE_OK) return rc;
+  }
+  return MCCE_OK;
+}
+
+extern "C" int mcce_reset(mcce_ctx* ctx, const int32_t* init_order, int keep_delta_stats, const float* delta_sum,
+                          int64_t delta_count) {
+  if (!ctx) return MCCE_EINVAL;
+  const mcce_config& c = ctx->cfg;
+  const size_t LS = (size_t)c.n_layers * c.n_streams, E = c.n_experts, C = c.cache_capacity, EW = ctx->EW;
+  if (delta_sum && delta_count < 0) return MCCE_EINVAL;
+  CK(cudaSetDevice(c.device));
+  CK(cudaDeviceSynchronize());
+  std::vector<uint32_t> stamp(LS * E, 0u), ever(LS * EW, 0u);
+  if (init_order) {
+    for (size_t p = 0; p < LS; ++p)
+      for (size_t r = 0; r < C; ++r) {
+        const int32_t e = init_order[p * C + r];
+        if (e < 0) continue;
+        if ((size_t)e >= E || stamp[p * E + e] != 0u) return MCCE_EINVAL;
+        if (r >= E) return MCCE_EINVAL;
+        stamp[p * E + e] = (uint32_t)(E - r);  // 1..E, below every later touch (> E); MRU largest
+        ever[p * EW + e / 32] |= 1u << (e % 32);
+      }
+  }
+  CK(cudaMemcpy(ctx->stamp, stamp.data(), stamp.size() * 4, cudaMemcpyHostToDevice));
+  CK(cudaMemcpy(ctx->ever, ever.data(), ever.size() * 4, cudaMemcpyHostToDevice));
+  CK(cudaMemset(ctx->miss, 0, LS * 4));
+  CK(cudaMemset(ctx->cold, 0, LS * 4));
+  CK(cudaMemset(ctx->err, 0, 64));
+  if (delta_sum) {
+    CK(cudaMemcpy(ctx->sum_range, delta_sum, LS * 4, cudaMemcpyHostToDevice));
+    ctx->delta_cnt = (uint64_t)delta_count;
+  } else if (!keep_delta_stats) {
+    CK(cudaMemset(ctx->sum_range, 0, LS * 4));
+    ctx->delta_cnt = 0;
+  }
+  ctx->tok = 0;
+  ctx->steps_since_reset = 0;
+  CK(cudaDeviceSynchronize());
+  return MCCE_OK;
+}
+
+extern "C" int mcce_route_step(mcce_ctx* ctx, int32_t n_steps, const void* hidden, const float* logits_in,
+                               int32_t* sel_idx, float* sel_w, float* logits_out, void* cuda_stream) {
+  if (!ctx || n_steps < 0 || !sel_idx || !sel_w) return MCCE_EINVAL;
+  if ((hidden == nullptr) == (logits_in == nullptr)) return MCCE_EINVAL;
+  const mcce_config& c = ctx->cfg;
+  if (hidden && !ctx->Wr) return MCCE_ESTATE;
+  if (c.delta_mode == MCCE_DELTA_FIXED && !ctx->fixed_delta) return MCCE_ESTATE;
+  if (n_steps == 0) return MCCE_OK;
+  // recency keys and the Delta count are 32-bit on the device
+  const uint64_t last_key = (uint64_t)c.n_experts + (ctx->tok + n_steps) * (uint64_t)c.top_k + c.top_k + 1;
+  if (last_key >= 0xffffffffull || ctx->delta_cnt + n_steps >= 0xffffffffull) return MCCE_ESTATE;
+  RouteParams p;
+  p.L = c.n_layers, p.S = c.n_streams, p.E = c.n_experts, p.K = c.top_k, p.J = c.top_j, p.C = c.cache_capacity;
+  p.d = c.d_model, p.n_steps = n_steps, p.lambda = c.lambda, p.delta_mode = c.delta_mode, p.renorm = c.renorm;
+  p.hidden_bf16 = c.hidden_dtype == MCCE_BF16;
+  p.hidden = hidden, p.logits_in = logits_in, p.Wr = ctx->Wr, p.fixed_delta = ctx->fixed_delta;
+  p.stamp = ctx->stamp, p.ever = ctx->ever, p.sum_range = ctx->sum_range, p.miss = ctx->miss, p.cold = ctx->cold;
+  p.sel_idx = sel_idx, p.sel_w = sel_w, p.logits_out = logits_out;
+  p.tok0 = (uint32_t)ctx->tok, p.cnt0 = (uint32_t)ctx->delta_cnt;
+  CK(launch_route(p, (cudaStream_t)cuda_stream));
+  ctx->tok += n_steps;
+  ctx->steps_since_reset += n_steps;
+  if (c.delta_mode == MCCE_DELTA_RUNNING) ctx->delta_cnt += n_steps;
+  return MCCE_OK;
+}
+
+extern "C" int mcce_moe_forward(mcce_ctx* ctx, const void* hidden, const int32_t* sel_idx, const float* sel_w,
+                                float* y, void* cuda_stream) {
+  if (!ctx || !hidden || !sel_idx || !sel_w || !y) return MCCE_EINVAL;
+  if (!ctx->Wg) return MCCE_ESTATE;
+  if (((uintptr_t)hidden % 16) || ((uintptr_t)y % 16)) return MCCE_EINVAL;
+  const mcce_config& c = ctx->cfg;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  GroupParams g;
+  g.L = c.n_layers, g.S = c.n_streams, g.E = c.n_experts, g.K = c.top_k;
+  g.sel_idx = sel_idx, g.offsets = ctx->offsets, g.perm = ctx->perm, g.inv = ctx->inv;
+  CK(launch_group(g, st));
+  const FfnParams f = ffn_params(ctx, hidden, sel_w, y);
+  CK(launch_gather(f, st));
+  if (ctx->use_tc) {
+    CK(tc_launch(ctx->tc, f, ctx->err, st));
+  } else {
+    CK(launch_ffn_simt(f, st));
+  }
+  CK(launch_combine(f, st));
+  return MCCE_OK;
+}
+
+extern "C" int mcce_decode_step_host(mcce_ctx* ctx, const void* hidden_host, float* y_host, int32_t* sel_idx_host,
+                                     void* cuda_stream) {
+  if (!ctx || !hidden_host || !y_host) return MCCE_EINVAL;
+  const mcce_config& c = ctx->cfg;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  const size_t LS = (size_t)c.n_layers * c.n_streams, esz = c.hidden_dtype == MCCE_BF16 ? 2 : 4;
+  CK(cudaMemcpyAsync(ctx->stage_hidden, hidden_host, LS * c.d_model * esz, cudaMemcpyHostToDevice, st));
+  int rc = mcce_route_step(ctx, 1, ctx->stage_hidden, nullptr, ctx->stage_sel, ctx->stage_w, nullptr, cuda_stream);
+  if (rc != MCCE_OK) return rc;
+  rc = mcce_moe_forward(ctx, ctx->stage_hidden, ctx->stage_sel, ctx->stage_w, ctx->stage_y, cuda_stream);
+  if (rc != MCCE_OK) return rc;
+  CK(cudaMemcpyAsync(y_host, ctx->stage_y, LS * c.d_model * 4, cudaMemcpyDeviceToHost, st));
+  if (sel_idx_host)
+    CK(cudaMemcpyAsync(sel_idx_host, ctx->stage_sel, LS * c.top_k * 4, cudaMemcpyDeviceToHost, st));
+  CK(cudaStreamSynchronize(st));
+  return MCCE_OK;
+}
+
+extern "C" int mcce_cache_stats(mcce_ctx* ctx, mcce_stats* total, mcce_stats* per_layer) {
+  if (!ctx || !total) return MCCE_EINVAL;
+  const mcce_config& c = ctx->cfg;
+  CK(cudaSetDevice(c.device));
+  CK(cudaDeviceSynchronize());
+  CK(launch_stats(ctx->miss, ctx->cold, ctx->stats_dev, c.n_layers, c.n_streams, 0));
+  std::vector<unsigned long long> h((size_t)c.n_layers * 2);
+  CK(cudaMemcpy(h.data(), ctx->stats_dev, h.size() * 8, cudaMemcpyDeviceToHost));
+  uint32_t err[4];
+  CK(cudaMemcpy(err, ctx->err, sizeof(err), cudaMemcpyDeviceToHost));
+  memset(total, 0, sizeof(*total));
+  for (int l = 0; l < c.n_layers; ++l) {
+    mcce_stats s;
+    s.steps = (int64_t)ctx->steps_since_reset * c.n_streams;
+    s.selections = s.steps * c.top_k;
+    s.misses = (int64_t)h[2 * l];
+    s.cold_misses = (int64_t)h[2 * l + 1];
+    if (per_layer) per_layer[l] = s;
+    total->steps += s.steps, total->selections += s.selections;
+    total->misses += s.misses, total->cold_misses += s.cold_misses;
+  }
+  return err[0] != 0 ? MCCE_ETIMEOUT : MCCE_OK;
+}
+
+extern "C" int mcce_get_cache_state(mcce_ctx* ctx, int32_t* order, uint8_t* ever, float* delta_sum,
+                                    int64_t* delta_count) {
+  if (!ctx || !order) return MCCE_EINVAL;
+  const mcce_config& c = ctx->cfg;
+  const size_t LS = (size_t)c.n_layers * c.n_streams, E = c.n_experts, C = c.cache_capacity, EW = ctx->EW;
+  CK(cudaSetDevice(c.device));
+  CK(cudaDeviceSynchronize());
+  std::vector<uint32_t> stamp(LS * E), ev(LS * EW);
+  CK(cudaMemcpy(stamp.data(), ctx->stamp, stamp.size() * 4, cudaMemcpyDeviceToHost));
+  CK(cudaMemcpy(ev.data(), ctx->ever, ev.size() * 4, cudaMemcpyDeviceToHost));
+  std::vector<std::pair<uint32_t, int32_t>> res;
+  for (size_t p = 0; p < LS; ++p) {
+    res.clear();
+    for (size_t e = 0; e < E; ++e)
+      if (stamp[p * E + e]) res.emplace_back(stamp[p * E + e], (int32_t)e);
+    // most recent (largest key) first; keys are unique
+    for (size_t a = 0; a < res.size(); ++a)
+      for (size_t b = a + 1; b < res.size(); ++b)
+        if (res[b].first > res[a].first) std::swap(res[a], res[b]);
+    for (size_t r = 0; r < C; ++r) order[p * C + r] = r < res.size() ? res[r].second : -1;
+    if (ever)
+      for (size_t e = 0; e < E; ++e) ever[p * E + e] = (ev[p * EW + e / 32] >> (e % 32)) & 1u;
+  }
+  if (delta_sum) CK(cudaMemcpy(delta_sum, ctx->sum_range, LS * 4, cudaMemcpyDeviceToHost));
+  if (delta_count) *delta_count = (int64_t)ctx->delta_cnt;
+  return MCCE_OK;
+}
+
+extern "C" int mcce_get_grouping(mcce_ctx* ctx, int32_t* offsets, int32_t* perm) {
+  if (!ctx || !offsets || !perm) return MCCE_EINVAL;
+  const mcce_config& c = ctx->cfg;
+  CK(cudaSetDevice(c.device));
+  CK(cudaDeviceSynchronize());
+  CK(cudaMemcpy(offsets, ctx->offsets, (size_t)c.n_layers * (c.n_experts + 1) * 4, cudaMemcpyDeviceToHost));
+  CK(cudaMemcpy(perm, ctx->perm, (size_t)c.n_layers * c.n_streams * c.top_k * 4, cudaMemcpyDeviceToHost));
+  return MCCE_OK;
+}
+
+extern "C" const char* mcce_strerror(int code) {
+  switch (code) {
+    case MCCE_OK: return "ok";
+    case MCCE_EINVAL: return "invalid argument or unsupported configuration";
+    case MCCE_ENOSPC: return "workspace too small";
+    case MCCE_ESTATE: return "weights not set, or a 32-bit recency counter would overflow (call mcce_reset)";
+    case MCCE_ECUDA: return "CUDA call failed (see mcce_last_cuda_error)";
+    case MCCE_ETIMEOUT: return "a bounded wait inside a kernel gave up";
+    default: return "unknown error";
+  }
+}
+
+extern "C" int mcce_last_cuda_error(const mcce_ctx* ctx) { return ctx ? ctx->last_cuda : 0; }

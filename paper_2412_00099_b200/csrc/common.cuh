@@ -1,0 +1,72 @@
+// Internal declarations shared by the translation units of libmcce.so.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "mcce.h"
+
+namespace mcce {
+
+constexpr int kMaxE = 256;
+constexpr int kMaxK = 16;
+
+// Everything the route kernel needs (passed by value).
+struct RouteParams {
+  int L, S, E, K, J, C, d;
+  int n_steps;
+  float lambda;
+  int delta_mode, renorm;
+  int hidden_bf16;
+  const void* hidden;        // [n_steps,L,S,d] or null
+  const float* logits_in;    // [n_steps,L,S,E] or null
+  const float* Wr;           // [L,E,d]
+  const float* fixed_delta;  // [L]
+  uint32_t* stamp;           // [L,S,E]   0 = not resident, else recency key
+  uint32_t* ever;            // [L,S,EW]  bit e%32 of word e/32
+  float* sum_range;          // [L,S]
+  uint32_t* miss;            // [L,S]
+  uint32_t* cold;            // [L,S]
+  int32_t* sel_idx;          // [n_steps,L,S,K]
+  float* sel_w;              // [n_steps,L,S,K]
+  float* logits_out;         // [n_steps,L,S,E] or null
+  uint32_t tok0;             // tokens already processed since the last reset
+  uint32_t cnt0;             // tokens already folded into the running Delta
+};
+
+struct GroupParams {
+  int L, S, E, K;
+  const int32_t* sel_idx;  // [L,S,K]
+  int32_t* offsets;        // [L,E+1]
+  int32_t* perm;           // [L,S*K] position -> pair
+  int32_t* inv;            // [L,S*K] pair -> position
+};
+
+// Rows of the activation / intermediate / output buffers: routed pairs first, [l][pos], then the
+// shared experts, [l][q][s].
+struct FfnParams {
+  int L, S, E, K, n_sh, d, I;
+  int bf16;
+  const void* hidden;  // [L,S,d]
+  const void *Wg, *Wu, *Wd, *shWg, *shWu, *shWd;
+  const int32_t* offsets;  // [L,E+1]
+  const int32_t* perm;     // [L,S*K]
+  const int32_t* inv;      // [L,S*K]
+  const float* sel_w;      // [L,S,K]
+  void* Xg;                // [L*S*K, d]   gathered activations, hidden dtype
+  void* H;                 // [rows, I]    silu(g)*u, weight dtype
+  float* O;                // [rows, d]    expert outputs
+  float* y;                // [L,S,d]
+};
+
+cudaError_t launch_route(const RouteParams& p, cudaStream_t st);
+cudaError_t launch_group(const GroupParams& p, cudaStream_t st);
+cudaError_t launch_gather(const FfnParams& p, cudaStream_t st);
+cudaError_t launch_ffn_simt(const FfnParams& p, cudaStream_t st);
+cudaError_t launch_combine(const FfnParams& p, cudaStream_t st);
+cudaError_t launch_stats(const uint32_t* miss, const uint32_t* cold, unsigned long long* out, int L, int S,
+                         cudaStream_t st);
+
+__device__ __forceinline__ float bf16_to_f32(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+}  // namespace mcce

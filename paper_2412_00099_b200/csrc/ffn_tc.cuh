@@ -1,0 +1,23 @@
+// Tensor-core (tcgen05 / TMEM / TMA) path of the grouped expert FFN: interface used by api.cu.
+#pragma once
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace mcce {
+
+// Everything prepared once per weight set: the TMA descriptors of the weight, activation and
+// intermediate tensors.  Plain data (the context is zero-initialised as a block of bytes).
+struct TcPlan {
+  alignas(64) CUtensorMap w_gate, w_up, w_down, sh_gate, sh_up, sh_down;  // weights, 128-row boxes
+  alignas(64) CUtensorMap x_routed, x_hidden, h_all;                      // activations, 16-row boxes
+  int ready;
+};
+
+bool tc_applicable(const mcce_config& c);
+int tc_plan(const mcce_config& c, const void* Wg, const void* Wu, const void* Wd, const void* shWg, const void* shWu,
+            const void* shWd, void* Xg, void* H, TcPlan* plan);
+// hidden changes from call to call, so its descriptor is (re)built here when the pointer changes.
+cudaError_t tc_launch(TcPlan& plan, const FfnParams& p, uint32_t* err_flag, cudaStream_t st);
+
+}  // namespace mcce

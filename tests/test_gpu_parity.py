@@ -1,0 +1,255 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle on the same seeded
+inputs.  Integer results (expert indices, cache states, counters, grouping) bit for bit; floating point
+within the stated tolerances."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2412_00099_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+if torch.cuda.is_available():
+    from paper_2412_00099_b200 import binding as mb
+    import helpers as H
+
+
+def ar1_logits(seed, T, L, S, E, rho=0.8, scale=1.5, quant=None):
+    """Synthetic router logits with temporal locality, drawn from the seeded generator."""
+    n = synth.normal(seed, synth.T_LOGITS, 0, 0, T * L * S * E).reshape(T, L, S, E)
+    z = np.empty_like(n)
+    h = n[0]
+    for t in range(T):
+        h = n[t] if t == 0 else np.float32(rho) * h + np.float32(np.sqrt(1 - rho * rho)) * n[t]
+        z[t] = np.float32(scale) * h
+    if quant:
+        z = (np.round(z / quant) * quant).astype(np.float32)   # exact ties, to exercise tie-breaking
+    return z
+
+
+# ---- generator -------------------------------------------------------------------------------------
+def test_generator_matches_host_definition_bit_for_bit():
+    words = mb.gen_philox_words(1000, seed=5, tensor_id=3, t=7, start_block=(1 << 32) - 500).cpu().numpy()
+    assert np.array_equal(words.view(np.uint32), synth.uint32_stream(5, 3, 7, (1 << 32) - 500, 1000))
+    for dtype in (torch.float32, torch.bfloat16):
+        out = torch.empty(100_003, dtype=dtype, device="cuda")
+        mb.gen_normal(out, seed=9, tensor_id=synth.T_WG, t=0, std=0.02, start=4096)
+        ref = synth.scaled_normal(9, synth.T_WG, 0, 4096, 100_003, 0.02, dtype == torch.bfloat16)
+        got = out.view(torch.int16).cpu().numpy().view(np.uint16) if dtype == torch.bfloat16 else out.cpu().numpy()
+        assert np.array_equal(got.view(ref.dtype), ref)
+    big = torch.empty(4_000_000, dtype=torch.float32, device="cuda")
+    mb.gen_normal(big, seed=1, tensor_id=synth.T_NOISE, t=3)
+    assert abs(big.mean().item()) < 2e-3 and abs(big.std().item() - 1) < 2e-3
+
+
+@pytest.mark.parametrize("wl", [synth.TINY, synth.QWEN.with_(L=2, S=3, d=64)])
+def test_hidden_trace_matches_host_definition(wl):
+    state = torch.empty(wl.L * wl.S * wl.d, dtype=torch.float32, device="cuda")
+    x = torch.empty((wl.L, wl.S, wl.d), dtype=torch.bfloat16 if wl.bf16 else torch.float32, device="cuda")
+    for t, ref in enumerate(wl.hidden_trace(12)):
+        mb.gen_hidden_step(state, x, wl.seed, t, wl.rho, wl.topic_offset)
+        got = x.view(torch.int16).cpu().numpy().view(np.uint16) if wl.bf16 else x.cpu().numpy()
+        assert np.array_equal(got, ref)
+
+
+# ---- routing from identical logits: bit-exact ---------------------------------------------------------
+ROUTE_CASES = [
+    # E,  K, J, C,  lam, delta_mode, renorm, quant
+    (8, 2, 1, 4, 0.5, 0, 1, None),
+    (8, 2, 1, 4, 0.0, 0, 1, None),
+    (8, 2, 1, 4, 1.0, 0, 0, 0.25),
+    (60, 4, 2, 30, 0.5, 0, 1, None),
+    (60, 4, 2, 15, 1.0, 1, 1, 0.125),
+    (64, 8, 2, 32, 0.5, 0, 1, 0.25),
+    (64, 6, 0, 24, 0.7, 0, 1, None),
+    (64, 6, 6, 24, 0.7, 0, 1, None),       # J = K
+    (33, 5, 1, 3, 0.9, 0, 1, None),        # C < K, E not a multiple of 32
+    (16, 2, 1, 1, 0.6, 0, 1, None),        # cache of one
+    (20, 3, 1, 20, 0.5, 0, 1, None),       # C = E
+    (12, 3, 1, 50, 0.5, 0, 1, None),       # C > E
+    (130, 7, 2, 40, 0.4, 0, 1, 0.5),       # five lanes-slots per lane, many ties
+    (256, 16, 3, 100, 0.3, 0, 1, None),    # maximum sizes
+    (1, 1, 0, 1, 0.5, 0, 1, None),         # degenerate: one expert
+    (5, 5, 2, 2, 2.5, 0, 1, None),         # K = E, lambda > 1
+]
+
+
+@pytest.mark.parametrize("E,K,J,C,lam,dm,renorm,quant", ROUTE_CASES)
+@pytest.mark.parametrize("chunk", [1, 7])
+def test_route_from_logits_is_bit_exact(E, K, J, C, lam, dm, renorm, quant, chunk):
+    L, S, T = 3, 19, 48          # S not a multiple of the CTA's stream block
+    wl = synth.TINY.with_(L=L, E=E, K=K, J=J, C=C, S=S, lam=lam, d=64, I=64)
+    fixed = np.linspace(2.0, 4.0, L).astype(np.float32) if dm else None
+    eng = mb.engine_for(wl, delta_mode=dm, renorm=renorm)
+    if dm:
+        eng.set_router(torch.zeros((L, E, 64), device="cuda"), H.to_dev(fixed))
+    o = H.oracle_for(wl, delta_mode=dm, renorm=renorm, fixed_delta=fixed)
+    z = ar1_logits(E * 131 + K, T, L, S, E, quant=quant)
+    H.check_route_exact(eng, o, z, chunk=chunk, check_every=3)
+    eng.close()
+
+
+def test_route_initial_state_and_resume():
+    wl = synth.TINY.with_(L=2, E=24, K=3, J=1, C=7, S=5, lam=0.5)
+    rng = np.random.default_rng(0)
+    init = np.full((wl.L, wl.S, wl.C), -1, np.int32)
+    for l in range(wl.L):
+        for s in range(wl.S):
+            n = int(rng.integers(0, wl.C + 1))
+            init[l, s, :n] = rng.choice(wl.E, n, replace=False)
+    z = ar1_logits(3, 40, wl.L, wl.S, wl.E)
+    eng, o = mb.engine_for(wl), H.oracle_for(wl)
+    eng.reset(init_order=init)
+    o.reset(init_order=init)
+    H.check_route_exact(eng, o, z[:20], chunk=4, check_every=1)
+    # export, rebuild a second engine from the exported state, continue: must stay identical
+    order, ever, dsum, cnt = eng.cache_state()
+    eng2 = mb.engine_for(wl)
+    eng2.reset(init_order=order, delta_sum=dsum, delta_count=cnt)
+    s1, w1 = eng.route_step(logits=H.to_dev(z[20:]), n_steps=20)
+    s2, w2 = eng2.route_step(logits=H.to_dev(z[20:]), n_steps=20)
+    assert torch.equal(s1, s2) and torch.equal(w1, w2)
+    assert np.array_equal(eng.cache_state()[0], eng2.cache_state()[0])
+    # and the first engine still tracks the oracle (the second lost only the 'ever' bits / counters)
+    for i in range(20):
+        osel, _ = o.route(z[20 + i])
+        assert np.array_equal(s1[i].cpu().numpy(), osel)
+    H.assert_state_equal(eng, o)
+
+
+def test_full_cache_only_cold_misses_on_gpu():
+    wl = synth.TINY.with_(L=2, E=16, K=4, J=1, C=16, S=9, lam=0.5)
+    eng = mb.engine_for(wl)
+    z = ar1_logits(11, 64, wl.L, wl.S, wl.E)
+    sel, _ = eng.route_step(logits=H.to_dev(z), n_steps=64)
+    total, _ = eng.cache_stats()
+    sel = sel.cpu().numpy()
+    distinct = sum(len(np.unique(sel[:, l, s])) for l in range(wl.L) for s in range(wl.S))
+    assert total[2] == total[3] == distinct and total[1] == 64 * wl.L * wl.S * wl.K
+
+
+# ---- routing from hidden states: follow mode -----------------------------------------------------------
+@pytest.mark.parametrize("lam", [0.0, 0.5, 1.0])
+def test_tiny_workload_end_to_end_routing(lam):
+    wl = synth.TINY.with_(lam=lam)
+    Wr = wl.router()
+    eng, o = mb.engine_for(wl), H.oracle_for(wl)
+    eng.set_router(H.to_dev(Wr))
+    steps, near, dz = H.check_route_follow(eng, o, Wr, wl.hidden_trace(wl.T), wl.bf16)
+    assert steps == wl.T * wl.S * wl.L
+    print("tiny lam=%.1f: %d steps, %d near ties, max logit err %.2e" % (lam, steps, near, dz))
+
+
+@pytest.mark.parametrize("base,kw", [
+    (synth.QWEN, dict(L=2, S=21, T=24)),
+    (synth.OLMOE, dict(L=2, S=16, T=16)),
+    (synth.DEEPSEEK, dict(L=1, S=10, T=16)),
+    (synth.MIXTRAL, dict(L=2, S=9, T=16)),
+    (synth.QWEN, dict(L=1, S=8, T=8, d=8200)),        # hidden size beyond one shared-memory chunk
+])
+def test_model_shaped_routing_from_hidden_states(base, kw):
+    kw = dict(kw)
+    T = kw.pop("T")
+    wl = base.with_(**kw)
+    Wr = wl.router()
+    eng, o = mb.engine_for(wl, ffn_impl=mb.FFN_SIMT), H.oracle_for(wl)
+    eng.set_router(H.to_dev(Wr))
+    steps, near, dz = H.check_route_follow(eng, o, Wr, wl.hidden_trace(T), wl.bf16)
+    print("%s: %d steps, %d near ties, max logit err %.2e" % (wl.name, steps, near, dz))
+
+
+# ---- grouping -------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("L,S,E,K", [(1, 4, 8, 2), (3, 256, 60, 4), (2, 512, 64, 8), (2, 37, 200, 5), (1, 1, 1, 1)])
+def test_grouping_is_the_stable_counting_sort(L, S, E, K):
+    wl = synth.TINY.with_(L=L, S=S, E=E, K=K, J=0, C=max(1, E // 2), d=64, I=64)
+    eng = mb.engine_for(wl)
+    W = {k: (None if v is None else H.to_dev(v)) for k, v in H.weights_for(wl).items()}
+    eng.set_experts(**W)
+    rng = np.random.default_rng(L * 1000 + S)
+    sel = np.stack([[rng.choice(E, K, replace=False) for _ in range(S)] for _ in range(L)]).astype(np.int32)
+    if E > 4:
+        sel[0, :, 0] = 1            # one very full bucket ...
+        sel[0][sel[0] == 3] = 0     # ... and one empty
+    x = torch.zeros((L, S, 64), device="cuda")
+    eng.moe_forward(x, H.to_dev(sel), torch.ones((L, S, K), device="cuda"))
+    offsets, perm = eng.grouping()
+    for l in range(L):
+        flat = sel[l].reshape(-1)
+        assert np.array_equal(offsets[l], np.concatenate([[0], np.cumsum(np.bincount(flat, minlength=E))]))
+        assert np.array_equal(perm[l], np.argsort(flat, kind="stable"))
+
+
+# ---- expert FFN ---------------------------------------------------------------------------------------
+def run_forward_case(wl, T, ffn_impl):
+    Wr = wl.router()
+    W = H.weights_for(wl)
+    eng, o = mb.engine_for(wl, ffn_impl=ffn_impl), H.oracle_for(wl)
+    eng.set_router(H.to_dev(Wr))
+    eng.set_experts(**{k: (None if v is None else H.to_dev(v)) for k, v in W.items()})
+    worst = (0.0, 0.0)
+    for x in wl.hidden_trace(T):
+        xd = H.to_dev(x)
+        sel, w, zg = eng.route_step(hidden=xd[None], want_logits=True)
+        y = eng.moe_forward(xd, sel[0], w[0]).cpu().numpy()
+        osel, ow = o.route(zg[0].cpu().numpy())
+        assert np.array_equal(sel[0].cpu().numpy(), osel)
+        # the oracle's FFN runs on the oracle's own selection and weights
+        y_ref = o.ffn(x, osel, ow, W["Wg"], W["Wu"], W["Wd"], W["shWg"], W["shWu"], W["shWd"])
+        e = H.ffn_close(y, y_ref)
+        worst = (max(worst[0], e[0]), max(worst[1], e[1]))
+    assert eng.cache_stats()[0] == tuple(o.stats()[0].tolist())
+    return worst
+
+
+def test_tiny_workload_forward_fp32():
+    worst = run_forward_case(synth.TINY.with_(T=32), 32, mb.FFN_SIMT)
+    print("tiny fp32 forward: max abs err %.2e" % worst[0])
+
+
+@pytest.mark.parametrize("base,kw", [
+    (synth.QWEN, dict(L=2, S=24, E=12, K=4, C=6, d=256, I=384, n_shared=2)),
+    (synth.MIXTRAL, dict(L=1, S=5, E=8, K=2, C=4, d=512, I=1032)),
+    (synth.OLMOE, dict(L=1, S=40, E=16, K=8, C=8, d=128, I=72)),
+])
+def test_model_shaped_forward_simt_bf16(base, kw):
+    worst = run_forward_case(base.with_(**kw), 3, mb.FFN_SIMT)
+    print("%s simt forward: max abs err %.2e" % (base.name, worst[0]))
+
+
+def test_decode_step_from_host_buffers():
+    wl = synth.QWEN.with_(L=2, S=16, E=12, K=4, C=6, d=256, I=256, n_shared=1)
+    Wr, W = wl.router(), H.weights_for(wl)
+    eng, ref = mb.engine_for(wl), mb.engine_for(wl)
+    for e in (eng, ref):
+        e.set_router(H.to_dev(Wr))
+        e.set_experts(**{k: (None if v is None else H.to_dev(v)) for k, v in W.items()})
+    xh = torch.empty((wl.L, wl.S, wl.d), dtype=torch.bfloat16).pin_memory()
+    yh = torch.empty((wl.L, wl.S, wl.d), dtype=torch.float32).pin_memory()
+    sh = torch.empty((wl.L, wl.S, wl.K), dtype=torch.int32).pin_memory()
+    for x in wl.hidden_trace(4):
+        xh.copy_(torch.from_numpy(x.view(np.int16)).view(torch.bfloat16))
+        eng.decode_step_host(xh, yh, sh)
+        xd = xh.cuda()
+        sel, w = ref.route_step(hidden=xd[None])
+        y = ref.moe_forward(xd, sel[0], w[0])
+        assert torch.equal(sh, sel[0].cpu()) and torch.equal(yh, y.cpu())
+
+
+# ---- argument checking: errors come back as codes, nothing is launched ------------------------------------
+def test_bad_arguments_are_rejected():
+    with pytest.raises(mb.McceError):
+        mb.Engine(L=1, E=300, K=2, J=1, n_shared=0, d=64, I=64, C_cap=4, S=4, lam=0.5)      # E too large
+    with pytest.raises(mb.McceError):
+        mb.Engine(L=1, E=8, K=2, J=3, n_shared=0, d=64, I=64, C_cap=4, S=4, lam=0.5)        # J > K
+    with pytest.raises(mb.McceError):
+        mb.Engine(L=1, E=8, K=2, J=1, n_shared=0, d=64, I=64, C_cap=4, S=4, lam=float("nan"))
+    eng = mb.engine_for(synth.TINY)
+    x = torch.zeros((1, 4, 64), device="cuda")
+    with pytest.raises(mb.McceError):
+        eng.route_step(hidden=x[None])                                                       # router not set
+    with pytest.raises(mb.McceError):
+        eng.moe_forward(x, torch.zeros((1, 4, 2), dtype=torch.int32, device="cuda"),
+                        torch.zeros((1, 4, 2), device="cuda"))                               # experts not set
+    lib = mb.load()
+    assert lib.mcce_route_step(eng.ctx, 1, None, None, None, None, None, None) == -1
+    assert lib.mcce_workspace_bytes(None) == 0
