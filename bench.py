@@ -1,0 +1,326 @@
+#!/usr/bin/env python
+"""Throughput of the cache-conditional MoE decode step on synthetic, model-shaped workloads.
+
+One "step" is one token of every (stream, layer): fused routing (router GEMV, softmax, cache-aware
+promotion, top-k, LRU update, miss counting), expert grouping, the grouped SwiGLU expert FFN and the
+weighted combine.  The metric is stream*token*layer steps per second.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload qwen] [--impl mcce|reference]
+
+Prints one JSON line (rank 0).  `--impl reference` times the plain CPU oracle on the host cores on a
+bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2412_00099_b200 import synth  # noqa: E402
+
+METRIC = "cache-aware MoE decode steps/s (stream*token*layer)"
+UNIT = "steps/s"
+FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu
+# capture summarised under profiles/ (None until captured for the current kernel).
+NCU_TRAFFIC_BYTES = None
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="qwen", choices=sorted(synth.ALIASES))
+    ap.add_argument("--cache", type=int, default=None, help="cache capacity C per (stream, layer)")
+    ap.add_argument("--lam", type=float, default=None, help="promotion strength lambda")
+    ap.add_argument("--impl", default="mcce", choices=["mcce", "reference"])
+    ap.add_argument("--ffn", default="auto", choices=["auto", "simt", "tensor"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    return ap.parse_args()
+
+
+def workload_of(args):
+    wl = synth.ALIASES[args.workload]
+    if args.cache is not None:
+        wl = wl.with_(C=args.cache)
+    if args.lam is not None:
+        wl = wl.with_(lam=args.lam)
+    return wl
+
+
+def config_of(wl, extra=None):
+    cfg = {"workload": wl.name, "streams": wl.S, "layers": wl.L, "experts": wl.E, "top_k": wl.K, "top_j": wl.J,
+           "shared_experts": wl.n_shared, "d_model": wl.d, "d_ff": wl.I, "cache_capacity": wl.C, "lambda": wl.lam,
+           "seed": wl.seed}
+    cfg.update(extra or {})
+    return cfg
+
+
+# ---------------------------------------------------------------------------------------------------
+# CPU oracle on a bounded sample (used by --impl reference and by the cpu_baseline key)
+def oracle_sample(wl, steps: int, warmup: int, core_seconds: float = 20.0):
+    """Times the oracle (routing + FFN, layer 0, the first S_s streams) on the host cores.
+    Returns (steps/s, threads, description, seconds per step)."""
+    from oracle import oracle as orc
+    threads = os.cpu_count() or 1
+    S_s = min(wl.S, max(4, threads))
+    sub = wl.with_(L=1, S=S_s)
+    # inputs of layer 0 from the seeded generator (identical to the full workload's)
+    Wr = sub.router()
+    W = {"Wg": sub.expert_tensor(synth.T_WG), "Wu": sub.expert_tensor(synth.T_WU), "Wd": sub.expert_tensor(synth.T_WD)}
+    sh = {}
+    for k, tid in (("shWg", synth.T_SH_WG), ("shWu", synth.T_SH_WU), ("shWd", synth.T_SH_WD)):
+        sh[k] = sub.expert_tensor(tid) if wl.n_shared else None
+    rows = [(0, s) for s in range(S_s)]
+    xs = [x.reshape(1, S_s, wl.d) for x in wl.hidden_trace(warmup + steps, rows=rows)]
+    o = orc.Oracle(orc.OracleConfig(1, wl.E, wl.K, wl.J, wl.n_shared, wl.d, wl.I, wl.C, S_s, wl.lam, 0, 1,
+                                    1 if wl.bf16 else 0), threads=threads)
+
+    def one(x):
+        z = o.logits(Wr, x)
+        sel, w = o.route(z)
+        return o.ffn(x, sel, w, W["Wg"], W["Wu"], W["Wd"], sh["shWg"], sh["shWu"], sh["shWd"])
+
+    for x in xs[:warmup]:
+        one(x)
+    t0 = time.perf_counter()
+    for x in xs[warmup:]:
+        one(x)
+    dt = time.perf_counter() - t0
+    desc = "layer 0, first %d of %d streams, %d tokens, routing + expert FFN, %d host threads" % (
+        S_s, wl.S, steps, threads)
+    return S_s * steps / dt, threads, desc, dt / steps
+
+
+def reference_arm(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    wl = workload_of(args)
+    # each step is one token of the sample; keep the whole run within a few minutes
+    steps, warmup = max(1, min(args.steps, 8)), max(0, min(args.warmup, 1))
+    value, threads, desc, sec = oracle_sample(wl, steps, warmup)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+            "warmup": warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": config_of(wl, {"sample": desc}),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ---------------------------------------------------------------------------------------------------
+class ClockSampler:
+    """nvidia-smi samples of the SM clock and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_id: str):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", gpu_id, "--query-gpu=" + self.Q,
+                                       "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.f,
+                                      stderr=subprocess.DEVNULL)
+        except OSError:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.p.kill()
+        self.f.flush()
+        rows = [r.split(",") for r in open(self.f.name).read().strip().splitlines() if r.count(",") >= 6]
+        os.unlink(self.f.name)
+        try:
+            sm = [float(r[0]) for r in rows]
+            out["sm_mhz"] = float(np.median(sm)) if sm else None
+            out["sm_max_mhz"] = float(rows[0][1]) if rows else None
+            out["power_w_max"] = max(float(r[2]) for r in rows) if rows else None
+            names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+            out["reasons"] = [n for i, n in enumerate(names) if any("Active" == r[3 + i].strip() for r in rows)]
+            out["samples"] = len(rows)
+        except (ValueError, IndexError):
+            pass
+        return out
+
+
+def measured_hbm_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            return float(json.load(open(path))["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+        except (KeyError, ValueError):
+            pass
+    return FALLBACK_HBM_GBS, "fallback (earlier pool measurement)"
+
+
+def main_arm(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2412_00099_b200 import binding as mb
+    from paper_2412_00099_b200.shard import replica_seed, reduce_max, reduce_sum
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path); use --impl reference for the oracle")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.device("cuda", local)
+
+    wl = workload_of(args)
+    # streams are independent: rank r owns its own S streams (weak scaling), distinguished by the seed
+    seed = replica_seed(wl.seed, rank)
+    ffn_impl = {"auto": mb.FFN_AUTO, "simt": mb.FFN_SIMT, "tensor": mb.FFN_TENSOR}[args.ffn]
+    eng = mb.engine_for(wl, ffn_impl=ffn_impl, device=local)
+    wdt = torch.bfloat16 if wl.bf16 else torch.float32
+
+    # ---- weights, generated on the device ------------------------------------------------------------
+    Wr = mb.gen_normal(torch.empty((wl.L, wl.E, wl.d), dtype=torch.float32, device=dev), seed, synth.T_ROUTER,
+                       std=wl.weight_std)
+    shp_up, shp_dn = (wl.L, wl.E, wl.I, wl.d), (wl.L, wl.E, wl.d, wl.I)
+    Wg = mb.gen_normal(torch.empty(shp_up, dtype=wdt, device=dev), seed, synth.T_WG, std=wl.weight_std)
+    Wu = mb.gen_normal(torch.empty(shp_up, dtype=wdt, device=dev), seed, synth.T_WU, std=wl.weight_std)
+    Wd = mb.gen_normal(torch.empty(shp_dn, dtype=wdt, device=dev), seed, synth.T_WD, std=wl.weight_std)
+    sh = [None, None, None]
+    if wl.n_shared:
+        for i, (tid, shp) in enumerate(((synth.T_SH_WG, (wl.L, wl.n_shared, wl.I, wl.d)),
+                                        (synth.T_SH_WU, (wl.L, wl.n_shared, wl.I, wl.d)),
+                                        (synth.T_SH_WD, (wl.L, wl.n_shared, wl.d, wl.I)))):
+            sh[i] = mb.gen_normal(torch.empty(shp, dtype=wdt, device=dev), seed, tid, std=wl.weight_std)
+    eng.set_router(Wr)
+    eng.set_experts(Wg, Wu, Wd, *sh)
+
+    # ---- hidden-state trace for warm-up + timed steps, resident in HBM ---------------------------------
+    W, K = args.warmup, args.steps
+    n_tok = W + K
+    hidden = torch.empty((n_tok, wl.L, wl.S, wl.d), dtype=wdt, device=dev)
+    state = torch.empty(wl.L * wl.S * wl.d, dtype=torch.float32, device=dev)
+    for t in range(n_tok):
+        mb.gen_hidden_step(state, hidden[t], seed, t, wl.rho, wl.topic_offset)
+    sel = torch.empty((1, wl.L, wl.S, wl.K), dtype=torch.int32, device=dev)
+    sw = torch.empty((1, wl.L, wl.S, wl.K), dtype=torch.float32, device=dev)
+    y = torch.empty((wl.L, wl.S, wl.d), dtype=torch.float32, device=dev)
+
+    def step(t):
+        eng.route_step(hidden=hidden[t], out=(sel, sw))
+        eng.moe_forward(hidden[t], sel[0], sw[0], out=y)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    for t in range(W):
+        step(t)
+    eng.profile(True)
+    eng.profile_read(reset=True)
+    barrier()
+    props = torch.cuda.get_device_properties(dev)
+    sampler = ClockSampler("GPU-" + str(props.uuid)) if hasattr(props, "uuid") else None
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for t in range(W, n_tok):
+        step(t)
+    e1.record()
+    barrier()
+    ms_total = reduce_max(e0.elapsed_time(e1), dev if world > 1 else None)
+    clocks = sampler.stop() if sampler else {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+    prof = eng.profile_read(reset=True)
+    eng.profile(False)
+
+    units_per_step = wl.S * wl.L                      # per rank
+    value = world * units_per_step * K / (ms_total * 1e-3)
+    total, _ = eng.cache_stats()
+    miss_rate = total[2] / max(1, total[1])
+    misses = reduce_sum(total[2], dev if world > 1 else None)
+    selections = reduce_sum(total[1], dev if world > 1 else None)
+
+    # ---- roofline of the dominant kernel (gate/up projection of the grouped expert FFN) ---------------
+    offsets, _ = eng.grouping()
+    touched = int((np.diff(offsets, axis=1) > 0).sum()) + wl.L * wl.n_shared
+    rows = wl.L * wl.S * (wl.K + wl.n_shared)
+    esz = 2 if wl.bf16 else 4
+    bytes_up = touched * 2 * wl.d * wl.I * esz + rows * wl.d * esz + rows * wl.I * esz
+    bytes_down = touched * wl.d * wl.I * esz + rows * wl.I * esz + rows * wl.d * 4
+    up_ms, up_n = prof["ffn_up"]
+    peak, peak_src = measured_hbm_peak()
+    achieved = bytes_up / (up_ms / max(1, up_n) * 1e-3) / 1e9
+    roofline = {"kernel": "ffn_up (H = silu(X Wg^T) * (X Wu^T), all expert groups)", "bound": "hbm",
+                "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
+                "traffic": NCU_TRAFFIC_BYTES, "algorithmic_bytes_per_launch": bytes_up,
+                "avg_launch_ms": up_ms / max(1, up_n)}
+    kernels = {k: {"ms_per_step": v[0] / K, "launches": v[1]} for k, v in prof.items()}
+    dn_ms, dn_n = prof["ffn_down"]
+    kernels["ffn_down"]["achieved_gbs"] = bytes_down / (dn_ms / max(1, dn_n) * 1e-3) / 1e9
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+            "ms_per_step": ms_total / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16" if wl.bf16 else "f32", "data": "synthetic",
+            "config": config_of(wl, {"l2": "inputs larger than L2: %.1f GB of expert weights streamed per step"
+                                           % ((bytes_up + bytes_down) / 1e9),
+                                     "ffn_path": "tensor" if _uses_tensor(eng) else "simt",
+                                     "experts_touched_per_step": touched}),
+            "miss_rate": misses / max(1, selections), "roofline": roofline, "kernels": kernels,
+            "gpu_launches": int(sum(v[1] for v in prof.values())), "clocks": clocks}
+
+    # ---- end to end through the host-buffer entry point -------------------------------------------------
+    if not args.no_e2e:
+        n_e2e = max(2, min(K, 10))
+        hh = torch.empty((n_e2e + 1, wl.L, wl.S, wl.d), dtype=wdt).pin_memory()
+        hh.copy_(hidden[:n_e2e + 1])
+        yh = torch.empty((wl.L, wl.S, wl.d), dtype=torch.float32).pin_memory()
+        eng.decode_step_host(hh[0], yh)
+        barrier()
+        t0 = time.perf_counter()
+        for t in range(1, n_e2e + 1):
+            eng.decode_step_host(hh[t], yh)
+        torch.cuda.synchronize(dev)
+        dt = reduce_max(time.perf_counter() - t0, dev if world > 1 else None)
+        line["e2e"] = {"value": world * units_per_step * n_e2e / dt, "unit": UNIT,
+                       "h2d_bytes_per_step": hh[0].numel() * hh.element_size(),
+                       "d2h_bytes_per_step": yh.numel() * 4, "steps": n_e2e,
+                       "call": "mcce_decode_step_host (pinned host buffers, copies inside the timed region)"}
+
+    # ---- the oracle on the host cores, beside it ------------------------------------------------------------
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        v, threads, desc, _ = oracle_sample(wl, steps=4, warmup=1)
+        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc}
+
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def _uses_tensor(eng):
+    return bool(eng.uses_tensor_path())
+
+
+if __name__ == "__main__":
+    a = parse_args()
+    if a.impl == "reference":
+        reference_arm(a)
+    else:
+        main_arm(a)

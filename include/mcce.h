@@ -154,6 +154,25 @@ int mcce_gen_hidden_step(float* state, void* x_out, int32_t dtype, uint64_t coun
 int mcce_gen_philox_words(uint32_t* out, uint64_t start_block, uint64_t n_blocks, uint32_t seed,
                           uint32_t tensor_id, uint32_t t, void* cuda_stream);
 
+/* Per-kernel device time, for measurement (no counterpart in the paper).  When enabled, every launch
+ * of this context is bracketed by a pair of CUDA events on its stream; mcce_profile_read waits for the
+ * recorded events and returns, per kernel kind, the summed milliseconds and the number of launches
+ * (HOST arrays of MCCE_N_KERNELS entries), clearing the sums if reset != 0. */
+enum {
+  MCCE_K_ROUTE = 0,    /* fused route kernel                         */
+  MCCE_K_GROUP = 1,    /* histogram + scan + scatter                 */
+  MCCE_K_GATHER = 2,   /* activation rows into expert order          */
+  MCCE_K_FFN_UP = 3,   /* H = silu(X Wg^T) * (X Wu^T), all groups    */
+  MCCE_K_FFN_DOWN = 4, /* O = H Wd^T, all groups                     */
+  MCCE_K_COMBINE = 5,  /* weighted sum over slots + shared experts   */
+  MCCE_N_KERNELS = 6
+};
+int mcce_profile(mcce_ctx* ctx, int enable);
+int mcce_profile_read(mcce_ctx* ctx, double* ms /*HOST*/, int64_t* launches /*HOST*/, int reset);
+
+/* 1 if mcce_moe_forward of this context runs the tcgen05/TMA expert kernels, 0 if the fp32-pipe ones. */
+int mcce_uses_tensor_path(const mcce_ctx* ctx);
+
 const char* mcce_strerror(int code);
 int mcce_last_cuda_error(const mcce_ctx* ctx); /* cudaError_t of the last failed CUDA call */
 

@@ -21,7 +21,7 @@ FFN_AUTO, FFN_SIMT, FFN_TENSOR = 0, 1, 2
 EXPORTS = [
     "mcce_workspace_bytes", "mcce_create", "mcce_destroy", "mcce_set_router", "mcce_set_experts", "mcce_reset",
     "mcce_route_step", "mcce_moe_forward", "mcce_decode_step_host", "mcce_cache_stats", "mcce_get_cache_state",
-    "mcce_get_grouping", "mcce_gen_normal", "mcce_gen_hidden_step", "mcce_gen_philox_words", "mcce_strerror",
+    "mcce_get_grouping", "mcce_profile", "mcce_profile_read", "mcce_uses_tensor_path", "mcce_gen_normal", "mcce_gen_hidden_step", "mcce_gen_philox_words", "mcce_strerror",
     "mcce_last_cuda_error",
 ]
 
@@ -68,6 +68,9 @@ def load():
         lib.mcce_cache_stats.argtypes = [vp, C.POINTER(Stats), C.POINTER(Stats)]
         lib.mcce_get_cache_state.argtypes = [vp, vp, vp, vp, C.POINTER(C.c_int64)]
         lib.mcce_get_grouping.argtypes = [vp, vp, vp]
+        lib.mcce_uses_tensor_path.argtypes = [vp]
+        lib.mcce_profile.argtypes = [vp, C.c_int]
+        lib.mcce_profile_read.argtypes = [vp, vp, vp, C.c_int]
         lib.mcce_gen_normal.argtypes = [vp, i32, u64, u64, u32, u32, u32, f32, vp]
         lib.mcce_gen_hidden_step.argtypes = [vp, vp, i32, u64, u32, u32, f32, f32, f32, vp]
         lib.mcce_gen_philox_words.argtypes = [vp, u64, u64, u32, u32, u32, vp]
@@ -208,6 +211,21 @@ class Engine:
         cnt = C.c_int64()
         _check(self.lib.mcce_get_cache_state(self.ctx, _ptr(order), _ptr(ever), _ptr(dsum), C.byref(cnt)), self.ctx)
         return order, ever, dsum, cnt.value
+
+    KERNELS = ("route", "group", "gather", "ffn_up", "ffn_down", "combine")
+
+    def uses_tensor_path(self) -> bool:
+        return self.lib.mcce_uses_tensor_path(self.ctx) == 1
+
+    def profile(self, enable: bool):
+        _check(self.lib.mcce_profile(self.ctx, int(enable)), self.ctx)
+
+    def profile_read(self, reset=True):
+        """{kernel: (total ms, launches)} from the CUDA events recorded around each launch."""
+        ms = np.zeros(len(self.KERNELS), np.float64)
+        n = np.zeros(len(self.KERNELS), np.int64)
+        _check(self.lib.mcce_profile_read(self.ctx, _ptr(ms), _ptr(n), int(reset)), self.ctx)
+        return {k: (float(ms[i]), int(n[i])) for i, k in enumerate(self.KERNELS)}
 
     def grouping(self):
         offsets = np.empty((self.L, self.E + 1), np.int32)

@@ -11,6 +11,8 @@
 
 using namespace mcce;
 
+constexpr int kMaxPairs = 1024;
+
 struct mcce_ctx {
   mcce_config cfg;
   int EW;
@@ -33,6 +35,13 @@ struct mcce_ctx {
   int last_cuda;
   int use_tc;
   TcPlan tc;
+  // optional per-kernel timing: event pairs recorded around each launch, summed by mcce_profile_read
+  int profiling;
+  int n_pairs;
+  cudaEvent_t ev[kMaxPairs][2];
+  int ev_kind[kMaxPairs];
+  double prof_ms[MCCE_N_KERNELS];
+  int64_t prof_launches[MCCE_N_KERNELS];
 };
 
 namespace {
@@ -105,6 +114,44 @@ int cuda_fail(mcce_ctx* ctx, cudaError_t e) {
     if (e_ != cudaSuccess) return cuda_fail(ctx, e_); \
   } while (0)
 
+// Folds the recorded event pairs into the per-kernel sums (synchronises on the last event).
+int drain_events(mcce_ctx* ctx) {
+  for (int i = 0; i < ctx->n_pairs; ++i) {
+    float ms = 0.f;
+    CK(cudaEventSynchronize(ctx->ev[i][1]));
+    CK(cudaEventElapsedTime(&ms, ctx->ev[i][0], ctx->ev[i][1]));
+    ctx->prof_ms[ctx->ev_kind[i]] += ms;
+    ctx->prof_launches[ctx->ev_kind[i]] += 1;
+  }
+  ctx->n_pairs = 0;
+  return MCCE_OK;
+}
+
+// Runs `launch` between two events on `st` when profiling is on.
+template <typename F>
+int timed(mcce_ctx* ctx, int kind, cudaStream_t st, F launch) {
+  if (!ctx->profiling) {
+    CK(launch());
+    return MCCE_OK;
+  }
+  if (ctx->n_pairs == kMaxPairs) {
+    const int rc = drain_events(ctx);
+    if (rc != MCCE_OK) return rc;
+  }
+  const int i = ctx->n_pairs;
+  CK(cudaEventRecord(ctx->ev[i][0], st));
+  CK(launch());
+  CK(cudaEventRecord(ctx->ev[i][1], st));
+  ctx->ev_kind[i] = kind;
+  ctx->n_pairs = i + 1;
+  return MCCE_OK;
+}
+#define TIMED(kind, st, expr)                                   \
+  do {                                                          \
+    const int rc_ = timed(ctx, kind, st, [&]() { return expr; }); \
+    if (rc_ != MCCE_OK) return rc_;                             \
+  } while (0)
+
 FfnParams ffn_params(const mcce_ctx* ctx, const void* hidden, const float* sel_w, float* y) {
   const mcce_config& c = ctx->cfg;
   FfnParams f;
@@ -157,6 +204,11 @@ extern "C" int mcce_create(const mcce_config* cfg, void* workspace, size_t works
 
 extern "C" int mcce_destroy(mcce_ctx* ctx) {
   if (!ctx) return MCCE_EINVAL;
+  if (ctx->profiling)
+    for (int i = 0; i < kMaxPairs; ++i) {
+      cudaEventDestroy(ctx->ev[i][0]);
+      cudaEventDestroy(ctx->ev[i][1]);
+    }
   delete ctx;
   return MCCE_OK;
 }
@@ -242,7 +294,7 @@ extern "C" int mcce_route_step(mcce_ctx* ctx, int32_t n_steps, const void* hidde
   p.stamp = ctx->stamp, p.ever = ctx->ever, p.sum_range = ctx->sum_range, p.miss = ctx->miss, p.cold = ctx->cold;
   p.sel_idx = sel_idx, p.sel_w = sel_w, p.logits_out = logits_out;
   p.tok0 = (uint32_t)ctx->tok, p.cnt0 = (uint32_t)ctx->delta_cnt;
-  CK(launch_route(p, (cudaStream_t)cuda_stream));
+  TIMED(MCCE_K_ROUTE, (cudaStream_t)cuda_stream, launch_route(p, (cudaStream_t)cuda_stream));
   ctx->tok += n_steps;
   ctx->steps_since_reset += n_steps;
   if (c.delta_mode == MCCE_DELTA_RUNNING) ctx->delta_cnt += n_steps;
@@ -259,15 +311,17 @@ extern "C" int mcce_moe_forward(mcce_ctx* ctx, const void* hidden, const int32_t
   GroupParams g;
   g.L = c.n_layers, g.S = c.n_streams, g.E = c.n_experts, g.K = c.top_k;
   g.sel_idx = sel_idx, g.offsets = ctx->offsets, g.perm = ctx->perm, g.inv = ctx->inv;
-  CK(launch_group(g, st));
+  TIMED(MCCE_K_GROUP, st, launch_group(g, st));
   const FfnParams f = ffn_params(ctx, hidden, sel_w, y);
-  CK(launch_gather(f, st));
+  TIMED(MCCE_K_GATHER, st, launch_gather(f, st));
   if (ctx->use_tc) {
-    CK(tc_launch(ctx->tc, f, ctx->err, st));
+    TIMED(MCCE_K_FFN_UP, st, tc_launch_up(ctx->tc, f, ctx->err, st));
+    TIMED(MCCE_K_FFN_DOWN, st, tc_launch_down(ctx->tc, f, ctx->err, st));
   } else {
-    CK(launch_ffn_simt(f, st));
+    TIMED(MCCE_K_FFN_UP, st, launch_ffn_simt_up(f, st));
+    TIMED(MCCE_K_FFN_DOWN, st, launch_ffn_simt_down(f, st));
   }
-  CK(launch_combine(f, st));
+  TIMED(MCCE_K_COMBINE, st, launch_combine(f, st));
   return MCCE_OK;
 }
 
@@ -348,6 +402,41 @@ extern "C" int mcce_get_grouping(mcce_ctx* ctx, int32_t* offsets, int32_t* perm)
   CK(cudaDeviceSynchronize());
   CK(cudaMemcpy(offsets, ctx->offsets, (size_t)c.n_layers * (c.n_experts + 1) * 4, cudaMemcpyDeviceToHost));
   CK(cudaMemcpy(perm, ctx->perm, (size_t)c.n_layers * c.n_streams * c.top_k * 4, cudaMemcpyDeviceToHost));
+  return MCCE_OK;
+}
+
+extern "C" int mcce_uses_tensor_path(const mcce_ctx* ctx) { return ctx ? ctx->use_tc : MCCE_EINVAL; }
+
+extern "C" int mcce_profile(mcce_ctx* ctx, int enable) {
+  if (!ctx) return MCCE_EINVAL;
+  CK(cudaSetDevice(ctx->cfg.device));
+  if (enable && !ctx->profiling) {
+    for (int i = 0; i < kMaxPairs; ++i) {
+      CK(cudaEventCreate(&ctx->ev[i][0]));
+      CK(cudaEventCreate(&ctx->ev[i][1]));
+    }
+    ctx->n_pairs = 0;
+  } else if (!enable && ctx->profiling) {
+    const int rc = drain_events(ctx);
+    if (rc != MCCE_OK) return rc;
+    for (int i = 0; i < kMaxPairs; ++i) {
+      cudaEventDestroy(ctx->ev[i][0]);
+      cudaEventDestroy(ctx->ev[i][1]);
+    }
+  }
+  ctx->profiling = enable != 0;
+  return MCCE_OK;
+}
+
+extern "C" int mcce_profile_read(mcce_ctx* ctx, double* ms, int64_t* launches, int reset) {
+  if (!ctx || !ms || !launches) return MCCE_EINVAL;
+  const int rc = drain_events(ctx);
+  if (rc != MCCE_OK) return rc;
+  for (int k = 0; k < MCCE_N_KERNELS; ++k) {
+    ms[k] = ctx->prof_ms[k];
+    launches[k] = ctx->prof_launches[k];
+    if (reset) ctx->prof_ms[k] = 0.0, ctx->prof_launches[k] = 0;
+  }
   return MCCE_OK;
 }
 

@@ -62,7 +62,8 @@ struct FfnParams {
 cudaError_t launch_route(const RouteParams& p, cudaStream_t st);
 cudaError_t launch_group(const GroupParams& p, cudaStream_t st);
 cudaError_t launch_gather(const FfnParams& p, cudaStream_t st);
-cudaError_t launch_ffn_simt(const FfnParams& p, cudaStream_t st);
+cudaError_t launch_ffn_simt_up(const FfnParams& p, cudaStream_t st);
+cudaError_t launch_ffn_simt_down(const FfnParams& p, cudaStream_t st);
 cudaError_t launch_combine(const FfnParams& p, cudaStream_t st);
 cudaError_t launch_stats(const uint32_t* miss, const uint32_t* cold, unsigned long long* out, int L, int S,
                          cudaStream_t st);

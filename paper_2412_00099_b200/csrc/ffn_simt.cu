@@ -138,16 +138,17 @@ __global__ void __launch_bounds__(kTB * 32) ffn_simt_kernel(const FfnParams p) {
   }
 }
 
-cudaError_t launch_ffn_simt(const FfnParams& p, cudaStream_t st) {
-  const int G = p.E + p.n_sh;
-  const dim3 ga((p.I + kTB * kRW - 1) / (kTB * kRW), p.L * G), gb((p.d + kTB * kRW - 1) / (kTB * kRW), p.L * G);
-  if (p.bf16) {
-    ffn_simt_kernel<__nv_bfloat16, true><<<ga, kTB * 32, 0, st>>>(p);
-    ffn_simt_kernel<__nv_bfloat16, false><<<gb, kTB * 32, 0, st>>>(p);
-  } else {
-    ffn_simt_kernel<float, true><<<ga, kTB * 32, 0, st>>>(p);
-    ffn_simt_kernel<float, false><<<gb, kTB * 32, 0, st>>>(p);
-  }
+cudaError_t launch_ffn_simt_up(const FfnParams& p, cudaStream_t st) {
+  const dim3 grid((p.I + kTB * kRW - 1) / (kTB * kRW), p.L * (p.E + p.n_sh));
+  if (p.bf16) ffn_simt_kernel<__nv_bfloat16, true><<<grid, kTB * 32, 0, st>>>(p);
+  else ffn_simt_kernel<float, true><<<grid, kTB * 32, 0, st>>>(p);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_ffn_simt_down(const FfnParams& p, cudaStream_t st) {
+  const dim3 grid((p.d + kTB * kRW - 1) / (kTB * kRW), p.L * (p.E + p.n_sh));
+  if (p.bf16) ffn_simt_kernel<__nv_bfloat16, false><<<grid, kTB * 32, 0, st>>>(p);
+  else ffn_simt_kernel<float, false><<<grid, kTB * 32, 0, st>>>(p);
   return cudaGetLastError();
 }
 

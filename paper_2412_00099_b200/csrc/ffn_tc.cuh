@@ -18,6 +18,7 @@ bool tc_applicable(const mcce_config& c);
 int tc_plan(const mcce_config& c, const void* Wg, const void* Wu, const void* Wd, const void* shWg, const void* shWu,
             const void* shWd, void* Xg, void* H, TcPlan* plan);
 // hidden changes from call to call, so its descriptor is (re)built here when the pointer changes.
-cudaError_t tc_launch(TcPlan& plan, const FfnParams& p, uint32_t* err_flag, cudaStream_t st);
+cudaError_t tc_launch_up(TcPlan& plan, const FfnParams& p, uint32_t* err_flag, cudaStream_t st);
+cudaError_t tc_launch_down(TcPlan& plan, const FfnParams& p, uint32_t* err_flag, cudaStream_t st);
 
 }  // namespace mcce

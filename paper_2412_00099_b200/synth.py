@@ -99,8 +99,24 @@ def _box_muller(xa, xb):
     return r * cx, r * sx
 
 
+_CHUNK = 1 << 20     # elements per work item when a large draw is split over host threads
+
+
 def normal(seed: int, tensor_id: int, t: int, start: int, count: int) -> np.ndarray:
     """Standard normals for flat elements [start, start+count) of tensor `tensor_id` at step t (fp32)."""
+    if count > 2 * _CHUNK and start % 4 == 0:
+        import os
+        from concurrent.futures import ThreadPoolExecutor
+        out = np.empty(count, np.float32)
+        pieces = [(o, min(_CHUNK, count - o)) for o in range(0, count, _CHUNK)]
+
+        def fill(piece):
+            o, n = piece
+            out[o:o + n] = normal(seed, tensor_id, t, start + o, n)
+
+        with ThreadPoolExecutor(os.cpu_count() or 1) as ex:
+            list(ex.map(fill, pieces))
+        return out
     b0, b1 = start // 4, (start + count + 3) // 4
     blocks = np.arange(b0, b1, dtype=np.uint64)
     x0, x1, x2, x3 = philox4x32_10(blocks & _MASK, blocks >> np.uint64(32), t, tensor_id, seed, 0)
