@@ -1,9 +1,458 @@
+// Grouped SwiGLU expert FFN of Eq. 1 on the 5th-generation tensor cores: a persistent, warp-specialised
+// weight streamer.
+//
+// At decode batch sizes every expert sees only tens of tokens, so the work is bound by streaming each
+// touched expert's weights from HBM exactly once.  The GEMMs are therefore "swapped": the weight rows
+// are the MMA M dimension (tiles of 128 rows), the expert's tokens are the N dimension (16..128 per
+// instruction), and the reduction runs over the hidden (gate/up) or intermediate (down) dimension:
+//
+//     up  :  G^T, U^T [128 x N] = Wg, Wu [128 x d] * X_e^T [d x N];   H = bf16(silu(G) * U)
+//     down:  O^T      [128 x N] = Wd     [128 x I] * H_e^T [I x N]
+//
+// One CTA per SM walks a static list of (layer, expert, 128-row tile) items.  Warp 0 issues TMA loads
+// (128B-swizzled 64-column slabs of the weight tile and of the token rows) into a ring of shared-memory
+// stages, warp 1 issues tcgen05.mma into one of two TMEM accumulator buffers, warps 2-5 drain the other
+// buffer with tcgen05.ld, apply the epilogue and write the result.  Every wait on an mbarrier is bounded:
+// on a timeout the CTA records an error word, stops, releases its TMEM and returns.
+#include <cuda.h>
+
 #include "ffn_tc.cuh"
 
 namespace mcce {
-bool tc_applicable(const mcce_config&) { return false; }
-int tc_plan(const mcce_config&, const void*, const void*, const void*, const void*, const void*, const void*, void*,
-            void*, TcPlan*) { return MCCE_EINVAL; }
-cudaError_t tc_launch_up(TcPlan&, const FfnParams&, uint32_t*, cudaStream_t) { return cudaErrorNotSupported; }
-cudaError_t tc_launch_down(TcPlan&, const FfnParams&, uint32_t*, cudaStream_t) { return cudaErrorNotSupported; }
+
+namespace {
+
+constexpr int kTileM = 128;   // weight rows per tile
+constexpr int kTileK = 64;    // reduction slab: 64 bf16 = one 128-byte swizzle row
+constexpr int kNMax = 128;    // tokens per pass over a weight tile
+constexpr int kXBox = 16;     // token rows per TMA box
+constexpr int kThreads = 192;
+constexpr uint32_t kABytes = kTileM * kTileK * 2;   // 16 KB
+constexpr uint32_t kBBytes = kNMax * kTileK * 2;    // 16 KB
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
+
+template <bool UP>
+struct Cfg {
+  static constexpr int kStages = UP ? 4 : 6;
+  static constexpr uint32_t kStageBytes = (UP ? 2 : 1) * kABytes + kBBytes;
+  static constexpr int kAccCols = UP ? 2 * kNMax : kNMax;   // TMEM columns per accumulator buffer
+  static constexpr int kTmemCols = 2 * kAccCols;            // two buffers: 512 / 256
+  static constexpr size_t kSmemBytes = (size_t)kStages * kStageBytes + 1024 /*align*/ + 256 /*barriers*/;
+};
+
+struct TcArgs {
+  int L, S, E, K, n_sh, d, I;
+  int n_items;
+  const int32_t* offsets;
+  __nv_bfloat16* H;
+  float* O;
+  uint32_t* err;
+};
+
+struct TcMaps {
+  CUtensorMap w0, w1, sw0, sw1;  // routed / shared weights (w1, sw1 only in the up kernel)
+  CUtensorMap x, xs;             // token rows of routed groups / of shared experts
+};
+
+// ---- PTX wrappers ------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+
+// Bounded wait.  Returns false if the CTA is aborting (this wait timed out, or another one did).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                          uint32_t* err, uint32_t code) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_ns();
+  for (uint32_t it = 1;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 255u) == 0u) {
+      if (*abort_flag) return false;
+      if (global_ns() - t0 > kWaitLimitNs) {
+        *abort_flag = 1u;
+        atomicCAS(err, 0u, code);
+        return false;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y)
+      : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t slot, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot), "r"(cols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// D[tmem] (+)= A[smem] * B[smem]^T, bf16 inputs, fp32 accumulate, one CTA.
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// Arrives on the mbarrier once every MMA issued so far by this thread has completed.
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// 16 consecutive fp32 columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes (64 bf16), 128B-swizzled:
+// 8-row groups 1024 bytes apart (stride byte offset), descriptor version 1, layout type SWIZZLE_128B.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
+  return (uint64_t)((addr & 0x3ffffu) >> 4) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor: fp32 accumulator, bf16 A and B, both K-major, M = 128, N = n.
+__device__ __forceinline__ uint32_t instr_desc(uint32_t n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((n >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+}
+
+// ---- the list of work items ----------------------------------------------------------------------------
+struct Item {
+  int m;          // tokens of the group
+  int wrow;       // first row of the 128-row weight tile in the weight tensor map
+  int xrow;       // first token row in the activation tensor map
+  size_t orow;    // first row of the group in H / O
+  int col0;       // first output column (= weight row inside the expert) of this tile
+  bool shared;
+};
+
+template <bool UP>
+__device__ __forceinline__ Item decode(const TcArgs& a, int w) {
+  const int rows = UP ? a.I : a.d;
+  const int RT = rows / kTileM, G = a.E + a.n_sh, P = a.S * a.K;
+  const int rt = w % RT, g = (w / RT) % G, l = w / (RT * G);
+  Item it;
+  it.col0 = rt * kTileM;
+  if (g < a.E) {
+    const int o0 = __ldg(a.offsets + (size_t)l * (a.E + 1) + g);
+    it.m = __ldg(a.offsets + (size_t)l * (a.E + 1) + g + 1) - o0;
+    it.shared = false;
+    it.wrow = (l * a.E + g) * rows + it.col0;
+    it.xrow = l * P + o0;
+    it.orow = (size_t)it.xrow;
+  } else {
+    const int q = g - a.E;
+    it.m = a.S;
+    it.shared = true;
+    it.wrow = (l * a.n_sh + q) * rows + it.col0;
+    it.orow = (size_t)a.L * P + (size_t)(l * a.n_sh + q) * a.S;
+    it.xrow = UP ? l * a.S : (int)it.orow;   // up: rows of the hidden tensor; down: rows of H
+  }
+  return it;
+}
+
+template <bool UP>
+__global__ void __launch_bounds__(kThreads, 1)
+ffn_tc_kernel(const __grid_constant__ TcMaps maps, const TcArgs a) {
+  using C = Cfg<UP>;
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_al = smem_raw + (smem_base - smem_u32(smem_raw));
+  uint64_t* bars = (uint64_t*)(smem_al + (size_t)C::kStages * C::kStageBytes);
+  // barrier slots: full[kStages], empty[kStages], tmem_full[2], tmem_empty[2]
+  const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * C::kStages;
+  const uint32_t bar_tfull = bar_empty + 8 * C::kStages, bar_tempty = bar_tfull + 16;
+  uint32_t* tmem_slot = (uint32_t*)(bars + 2 * C::kStages + 4);
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int R = UP ? a.d : a.I;       // reduction length
+  const int KT = R / kTileK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < C::kStages; ++s) {
+      mbar_init(bar_full + 8 * s, 1);
+      mbar_init(bar_empty + 8 * s, 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(bar_tfull + 8 * b, 1);
+      mbar_init(bar_tempty + 8 * b, 4);
+    }
+    *abort_flag = 0u;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) tmem_alloc(smem_u32(tmem_slot), C::kTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ---- TMA producer --------------------------------------------------------------------------------
+    if (lane == 0) {
+      uint32_t stage = 0, phase = 0;
+      bool alive = true;
+      for (int w = blockIdx.x; w < a.n_items && alive; w += gridDim.x) {
+        const Item it = decode<UP>(a, w);
+        const CUtensorMap* mw0 = it.shared ? &maps.sw0 : &maps.w0;
+        const CUtensorMap* mw1 = it.shared ? &maps.sw1 : &maps.w1;
+        const CUtensorMap* mx = it.shared ? &maps.xs : &maps.x;
+        for (int c0 = 0; c0 < it.m && alive; c0 += kNMax) {
+          const int n = (min(kNMax, it.m - c0) + 15) & ~15;
+          const uint32_t tx = (UP ? 2 : 1) * kABytes + (uint32_t)n * kTileK * 2;
+          for (int kt = 0; kt < KT; ++kt) {
+            if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, a.err, 1u)) {
+              alive = false;
+              break;
+            }
+            const uint32_t sa = smem_base + stage * C::kStageBytes;
+            const uint32_t full = bar_full + 8 * stage;
+            mbar_expect_tx(full, tx);
+            tma_load_2d(sa, mw0, kt * kTileK, it.wrow, full);
+            if (UP) tma_load_2d(sa + kABytes, mw1, kt * kTileK, it.wrow, full);
+            const uint32_t sb = sa + (UP ? 2 : 1) * kABytes;
+            for (int j = 0; j < n; j += kXBox)
+              tma_load_2d(sb + j * kTileK * 2, mx, kt * kTileK, it.xrow + c0 + j, full);
+            if (++stage == C::kStages) stage = 0, phase ^= 1u;
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---- MMA issuer ------------------------------------------------------------------------------------
+    if (lane == 0) {
+      uint32_t stage = 0, phase = 0, acc_iter = 0;
+      bool alive = true;
+      for (int w = blockIdx.x; w < a.n_items && alive; w += gridDim.x) {
+        const Item it = decode<UP>(a, w);
+        for (int c0 = 0; c0 < it.m && alive; c0 += kNMax, ++acc_iter) {
+          const uint32_t n = (uint32_t)(min(kNMax, it.m - c0) + 15) & ~15u;
+          const uint32_t idesc = instr_desc(n);
+          const uint32_t buf = acc_iter & 1u, acc_phase = (acc_iter >> 1) & 1u;
+          if (!mbar_wait(bar_tempty + 8 * buf, acc_phase ^ 1u, abort_flag, a.err, 2u)) {
+            alive = false;
+            break;
+          }
+          tc_fence_after();
+          const uint32_t d0 = tmem_base + buf * C::kAccCols;
+          for (int kt = 0; kt < KT; ++kt) {
+            if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag, a.err, 3u)) {
+              alive = false;
+              break;
+            }
+            tc_fence_after();
+            const uint32_t sa = smem_base + stage * C::kStageBytes;
+            const uint32_t sb = sa + (UP ? 2 : 1) * kABytes;
+#pragma unroll
+            for (int k = 0; k < kTileK / 16; ++k) {
+              const uint32_t acc = (kt > 0 || k > 0) ? 1u : 0u;
+              const uint64_t bd = smem_desc(sb + k * 32);
+              umma_bf16(d0, smem_desc(sa + k * 32), bd, idesc, acc);
+              if (UP) umma_bf16(d0 + kNMax, smem_desc(sa + kABytes + k * 32), bd, idesc, acc);
+            }
+            umma_commit(bar_empty + 8 * stage);   // frees the stage once these MMAs have read it
+            if (++stage == C::kStages) stage = 0, phase ^= 1u;
+          }
+          if (alive) umma_commit(bar_tfull + 8 * buf);
+        }
+      }
+    }
+  } else {
+    // ---- epilogue warps: TMEM -> registers -> global ---------------------------------------------------
+    const int quad = warp & 3;                         // TMEM lane quadrant this warp may read
+    const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+    uint32_t acc_iter = 0;
+    bool alive = true;
+    for (int w = blockIdx.x; w < a.n_items && alive; w += gridDim.x) {
+      const Item it = decode<UP>(a, w);
+      const int col = it.col0 + quad * 32 + lane;      // output feature handled by this thread
+      for (int c0 = 0; c0 < it.m && alive; c0 += kNMax, ++acc_iter) {
+        const int ntok = min(kNMax, it.m - c0);
+        const int n = (ntok + 15) & ~15;
+        const uint32_t buf = acc_iter & 1u, acc_phase = (acc_iter >> 1) & 1u;
+        if (!mbar_wait(bar_tfull + 8 * buf, acc_phase, abort_flag, a.err, 4u)) {
+          alive = false;
+          break;
+        }
+        tc_fence_after();
+        const uint32_t t0 = tmem_base + lane_addr + buf * C::kAccCols;
+        for (int n0 = 0; n0 < n; n0 += 16) {
+          float g[16];
+          tmem_ld16(t0 + n0, g);
+          if (UP) {
+            float u[16];
+            tmem_ld16(t0 + kNMax + n0, u);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              if (n0 + j < ntok) {
+                const float h = __fdividef(g[j], 1.f + __expf(-g[j])) * u[j];
+                a.H[(it.orow + c0 + n0 + j) * a.I + col] = __float2bfloat16_rn(h);
+              }
+            }
+          } else {
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 16; ++j)
+              if (n0 + j < ntok) a.O[(it.orow + c0 + n0 + j) * a.d + col] = g[j];
+          }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);
+      }
+    }
+  }
+
+  // ---- teardown ----------------------------------------------------------------------------------------
+  __syncwarp();
+  if (*abort_flag) {
+    // give copies and MMAs still in flight time to land before shared memory and TMEM are released
+    const unsigned long long t0 = global_ns();
+    while (global_ns() - t0 < 200000ull) __nanosleep(1000);
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (warp == 1) tmem_dealloc(tmem_base, C::kTmemCols);
+}
+
+// ---- host side -------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                             const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                             CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeFn encode_fn() {
+  static EncodeFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = (EncodeFn)p;
+  }
+  return fn;
+}
+
+// bf16 matrix [rows, cols] row-major; boxes of [box_rows, 64 columns], 128-byte swizzle, zero fill.
+bool make_map(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+  EncodeFn fn = encode_fn();
+  if (!fn || !base) return false;
+  const cuuint64_t dims[2] = {cols, rows};
+  const cuuint64_t strides[1] = {cols * 2};
+  const cuuint32_t box[2] = {(cuuint32_t)kTileK, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <bool UP>
+cudaError_t launch(const TcMaps& maps, const FfnParams& p, uint32_t* err, cudaStream_t st) {
+  static int sms = 0;
+  if (!sms) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    cudaError_t e = cudaFuncSetAttribute(ffn_tc_kernel<UP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)Cfg<UP>::kSmemBytes);
+    if (e != cudaSuccess) {
+      sms = 0;
+      return e;
+    }
+  }
+  TcArgs a;
+  a.L = p.L, a.S = p.S, a.E = p.E, a.K = p.K, a.n_sh = p.n_sh, a.d = p.d, a.I = p.I;
+  a.n_items = p.L * (p.E + p.n_sh) * ((UP ? p.I : p.d) / kTileM);
+  a.offsets = p.offsets, a.H = (__nv_bfloat16*)p.H, a.O = p.O, a.err = err;
+  const int grid = a.n_items < sms ? a.n_items : sms;
+  ffn_tc_kernel<UP><<<grid, kThreads, Cfg<UP>::kSmemBytes, st>>>(maps, a);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+bool tc_applicable(const mcce_config& c) {
+  return c.hidden_dtype == MCCE_BF16 && c.weight_dtype == MCCE_BF16 && c.d_model % kTileM == 0 &&
+         c.d_ff % kTileM == 0;
+}
+
+int tc_plan(const mcce_config& c, const void* Wg, const void* Wu, const void* Wd, const void* shWg, const void* shWu,
+            const void* shWd, void* Xg, void* H, TcPlan* plan) {
+  const uint64_t L = c.n_layers, E = c.n_experts, S = c.n_streams, K = c.top_k, nsh = c.n_shared;
+  const uint64_t d = c.d_model, I = c.d_ff;
+  const uint64_t rows = L * S * K + L * nsh * S;
+  bool ok = make_map(&plan->w_gate, Wg, L * E * I, d, kTileM) && make_map(&plan->w_up, Wu, L * E * I, d, kTileM) &&
+            make_map(&plan->w_down, Wd, L * E * d, I, kTileM);
+  if (nsh)
+    ok = ok && make_map(&plan->sh_gate, shWg, L * nsh * I, d, kTileM) &&
+         make_map(&plan->sh_up, shWu, L * nsh * I, d, kTileM) && make_map(&plan->sh_down, shWd, L * nsh * d, I, kTileM);
+  ok = ok && make_map(&plan->x_routed, Xg, L * S * K + 256, d, kXBox) && make_map(&plan->h_all, H, rows + 256, I, kXBox);
+  plan->hidden_ptr = nullptr;
+  plan->ready = ok;
+  return ok ? MCCE_OK : MCCE_ECUDA;
+}
+
+cudaError_t tc_launch_up(TcPlan& plan, const FfnParams& p, uint32_t* err_flag, cudaStream_t st) {
+  if (!plan.ready) return cudaErrorNotReady;
+  if (p.n_sh && plan.hidden_ptr != p.hidden) {
+    if (!make_map(&plan.x_hidden, p.hidden, (uint64_t)p.L * p.S, p.d, kXBox)) return cudaErrorInvalidValue;
+    plan.hidden_ptr = p.hidden;
+  }
+  TcMaps m;
+  m.w0 = plan.w_gate, m.w1 = plan.w_up, m.x = plan.x_routed;
+  m.sw0 = p.n_sh ? plan.sh_gate : plan.w_gate, m.sw1 = p.n_sh ? plan.sh_up : plan.w_up;
+  m.xs = p.n_sh ? plan.x_hidden : plan.x_routed;
+  return launch<true>(m, p, err_flag, st);
+}
+
+cudaError_t tc_launch_down(TcPlan& plan, const FfnParams& p, uint32_t* err_flag, cudaStream_t st) {
+  if (!plan.ready) return cudaErrorNotReady;
+  TcMaps m;
+  m.w0 = plan.w_down, m.w1 = plan.w_down, m.x = plan.h_all, m.xs = plan.h_all;
+  m.sw0 = p.n_sh ? plan.sh_down : plan.w_down, m.sw1 = m.sw0;
+  return launch<false>(m, p, err_flag, st);
+}
+
 }  // namespace mcce

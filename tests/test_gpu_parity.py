@@ -216,6 +216,44 @@ def test_model_shaped_forward_simt_bf16(base, kw):
     print("%s simt forward: max abs err %.2e" % (base.name, worst[0]))
 
 
+TC_CASES = [
+    (synth.QWEN, dict(L=2, S=24, E=12, K=4, C=6, d=256, I=384, n_shared=2)),      # small groups, empty groups
+    (synth.QWEN, dict(L=1, S=300, E=4, K=2, C=2, d=128, I=128, n_shared=1)),      # > 128 tokens per expert: chunks
+    (synth.OLMOE, dict(L=2, S=77, E=16, K=8, C=8, d=384, I=256)),                 # ragged token counts
+    (synth.MIXTRAL, dict(L=1, S=19, E=8, K=2, C=4, d=1024, I=2048)),              # long reductions, many stages
+    (synth.DEEPSEEK, dict(L=3, S=33, E=64, K=6, C=24, d=256, I=128, n_shared=2)),  # many experts, most nearly empty
+]
+
+
+@pytest.mark.parametrize("base,kw", TC_CASES)
+def test_model_shaped_forward_tensor_core_bf16(base, kw):
+    wl = base.with_(**kw)
+    eng = mb.engine_for(wl, ffn_impl=mb.FFN_TENSOR)
+    assert eng.uses_tensor_path()
+    eng.close()
+    worst = run_forward_case(wl, 3, mb.FFN_TENSOR)
+    print("%s tensor-core forward: max abs err %.2e" % (base.name, worst[0]))
+
+
+def test_tensor_core_path_agrees_with_simt_path():
+    """Same inputs through both expert-FFN implementations of the library (a consistency check on
+    top of the oracle comparisons above)."""
+    wl = synth.QWEN.with_(L=2, S=64, E=20, K=4, C=10, d=512, I=640, n_shared=1)
+    W = {k: (None if v is None else H.to_dev(v)) for k, v in H.weights_for(wl).items()}
+    x = H.to_dev(next(iter(wl.hidden_trace(1))))
+    rng = np.random.default_rng(1)
+    sel = H.to_dev(np.stack([[rng.choice(wl.E, wl.K, replace=False) for _ in range(wl.S)]
+                             for _ in range(wl.L)]).astype(np.int32))
+    w = torch.rand((wl.L, wl.S, wl.K), device="cuda")
+    ys = []
+    for impl in (mb.FFN_SIMT, mb.FFN_TENSOR):
+        eng = mb.engine_for(wl, ffn_impl=impl)
+        eng.set_experts(**W)
+        ys.append(eng.moe_forward(x, sel, w).cpu().numpy())
+        eng.cache_stats()
+    H.ffn_close(ys[1], ys[0])
+
+
 def test_decode_step_from_host_buffers():
     wl = synth.QWEN.with_(L=2, S=16, E=12, K=4, C=6, d=256, I=256, n_shared=1)
     Wr, W = wl.router(), H.weights_for(wl)
