@@ -38,11 +38,13 @@ NCU_TRAFFIC_BYTES = None
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="qwen", choices=sorted(synth.ALIASES))
     ap.add_argument("--cache", type=int, default=None, help="cache capacity C per (stream, layer)")
     ap.add_argument("--lam", type=float, default=None, help="promotion strength lambda")
+    ap.add_argument("--layers", type=int, default=None,
+                    help="fewer layers than the workload has (small cases for profiler captures; not a bench line)")
     ap.add_argument("--impl", default="mcce", choices=["mcce", "reference"])
     ap.add_argument("--ffn", default="auto", choices=["auto", "simt", "tensor"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -56,6 +58,8 @@ def workload_of(args):
         wl = wl.with_(C=args.cache)
     if args.lam is not None:
         wl = wl.with_(lam=args.lam)
+    if args.layers is not None:
+        wl = wl.with_(L=args.layers, name=wl.name + "[%d layers]" % args.layers)
     return wl
 
 
@@ -215,6 +219,9 @@ def main_arm(args):
     # ---- hidden-state trace for warm-up + timed steps, resident in HBM ---------------------------------
     W, K = args.warmup, args.steps
     n_tok = W + K
+    per_tok = wl.L * wl.S * wl.d * (2 if wl.bf16 else 4)
+    if n_tok * per_tok > 24e9:
+        raise SystemExit("hidden trace of %d tokens does not fit the budget; use fewer steps" % n_tok)
     hidden = torch.empty((n_tok, wl.L, wl.S, wl.d), dtype=wdt, device=dev)
     state = torch.empty(wl.L * wl.S * wl.d, dtype=torch.float32, device=dev)
     for t in range(n_tok):
