@@ -30,9 +30,10 @@ from paper_2412_00099_b200 import synth  # noqa: E402
 METRIC = "cache-aware MoE decode steps/s (stream*token*layer)"
 UNIT = "steps/s"
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu
-# capture summarised under profiles/ (None until captured for the current kernel).
-NCU_TRAFFIC_BYTES = None
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel (ffn_up), per layer,
+# from the ncu capture summarised in profiles/ffn_tc_kernel_qwen_4layers.md (a 4-layer case; traffic
+# grows in proportion to the layer count).  Workloads without a capture of the current kernel: None.
+NCU_TRAFFIC_BYTES_PER_LAYER = {"qwen1.5-moe-a2.7b-shaped": (3.155721e9 + 24.963072e6) / 4}
 
 
 def parse_args():
@@ -276,7 +277,9 @@ def main_arm(args):
     achieved = bytes_up / (up_ms / max(1, up_n) * 1e-3) / 1e9
     roofline = {"kernel": "ffn_up (H = silu(X Wg^T) * (X Wu^T), all expert groups)", "bound": "hbm",
                 "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
-                "traffic": NCU_TRAFFIC_BYTES, "algorithmic_bytes_per_launch": bytes_up,
+                "traffic": (NCU_TRAFFIC_BYTES_PER_LAYER[synth.ALIASES[args.workload].name] * wl.L
+                            if _uses_tensor(eng) and synth.ALIASES[args.workload].name in NCU_TRAFFIC_BYTES_PER_LAYER
+                            and args.cache is None else None), "algorithmic_bytes_per_launch": bytes_up,
                 "avg_launch_ms": up_ms / max(1, up_n)}
     kernels = {k: {"ms_per_step": v[0] / K, "launches": v[1]} for k, v in prof.items()}
     dn_ms, dn_n = prof["ffn_down"]
