@@ -33,7 +33,8 @@ enum {
   MCCE_ENOSPC = -2,   /* workspace too small                                            */
   MCCE_ESTATE = -3,   /* weights not set, or a counter would overflow (reset needed)    */
   MCCE_ECUDA = -4,    /* a CUDA call failed; see mcce_last_cuda_error                   */
-  MCCE_ETIMEOUT = -5  /* a bounded wait inside a kernel gave up; the context stays usable */
+  MCCE_ETIMEOUT = -5, /* a bounded wait inside a kernel gave up; the context stays usable */
+  MCCE_ELIMIT = -6    /* problem larger than the fixed array of mcce_route_trace_static   */
 };
 
 enum { MCCE_F32 = 0, MCCE_BF16 = 1 };
@@ -169,6 +170,35 @@ enum {
 };
 int mcce_profile(mcce_ctx* ctx, int enable);
 int mcce_profile_read(mcce_ctx* ctx, double* ms /*HOST*/, int64_t* launches /*HOST*/, int reset);
+
+/* Routing with no context, no workspace and no allocation of any kind.  The paper has no counterpart
+ * to this call; it exists for callers that cannot allocate device memory where they need routing
+ * decisions: a server whose memory pool already owns the whole GPU, a plug-in that only receives input
+ * and output buffers, or a latency-critical callback that must not enter the allocator.
+ *
+ * Runs the same fused route kernel as mcce_route_step over n_steps tokens of every (stream, layer),
+ * starting from EMPTY caches, zero counters and (running mode) an empty Delta statistic.  The cache
+ * state it needs while it runs lives in a fixed array inside the library image
+ * (mcce_route_trace_static_limit() bytes = 4 MiB, resident on every GPU that loads the library until
+ * the process exits) instead of in a workspace.  The state needs about L*S*(4*E + 4*ceil(E/32) + 12)
+ * bytes; a configuration that does not fit is refused with MCCE_ELIMIT and nothing is launched.
+ *   cfg         HOST; n_layers, n_streams, n_experts, top_k, top_j, cache_capacity, lambda,
+ *               delta_mode, renorm, hidden_dtype and d_model are used, the rest is ignored
+ *   hidden, Wr  DEVICE [n_steps,L,S,d] (hidden_dtype) and fp32 [L,E,d], or both NULL
+ *   logits_in   DEVICE fp32 [n_steps,L,S,E], or NULL; exactly one of hidden / logits_in is given
+ *   fixed_delta DEVICE fp32 [L], only for MCCE_DELTA_FIXED
+ *   sel_idx, sel_w  DEVICE outputs [n_steps,L,S,K], as in mcce_route_step
+ *   totals_host HOST, optional: Eq. 4 counters summed over everything; asking for them makes the call
+ *               wait for the stream, otherwise it only enqueues work
+ * The device that is current when the call is made is used.  The first call on each device looks up
+ * the array's device address; make that first call outside any stream capture.  The call uses no
+ * cudaMalloc / cudaFree and no allocating library routine.  Every call on a device shares the one
+ * array and first clears the part it uses, so nothing carries over between calls -- and two calls
+ * whose GPU work overlaps (different streams, or different host threads) race on it: serialise them. */
+size_t mcce_route_trace_static_limit(void);
+int mcce_route_trace_static(const mcce_config* cfg /*HOST*/, int32_t n_steps, const void* hidden, const float* Wr,
+                            const float* logits_in, const float* fixed_delta, int32_t* sel_idx, float* sel_w,
+                            mcce_stats* totals_host, void* cuda_stream);
 
 /* 1 if mcce_moe_forward of this context runs the tcgen05/TMA expert kernels, 0 if the fp32-pipe ones. */
 int mcce_uses_tensor_path(const mcce_ctx* ctx);

@@ -21,7 +21,8 @@ FFN_AUTO, FFN_SIMT, FFN_TENSOR = 0, 1, 2
 EXPORTS = [
     "mcce_workspace_bytes", "mcce_create", "mcce_destroy", "mcce_set_router", "mcce_set_experts", "mcce_reset",
     "mcce_route_step", "mcce_moe_forward", "mcce_decode_step_host", "mcce_cache_stats", "mcce_get_cache_state",
-    "mcce_get_grouping", "mcce_profile", "mcce_profile_read", "mcce_uses_tensor_path", "mcce_gen_normal", "mcce_gen_hidden_step", "mcce_gen_philox_words", "mcce_strerror",
+    "mcce_get_grouping", "mcce_profile", "mcce_profile_read", "mcce_uses_tensor_path", "mcce_route_trace_static",
+    "mcce_route_trace_static_limit", "mcce_gen_normal", "mcce_gen_hidden_step", "mcce_gen_philox_words", "mcce_strerror",
     "mcce_last_cuda_error",
 ]
 
@@ -69,6 +70,8 @@ def load():
         lib.mcce_get_cache_state.argtypes = [vp, vp, vp, vp, C.POINTER(C.c_int64)]
         lib.mcce_get_grouping.argtypes = [vp, vp, vp]
         lib.mcce_uses_tensor_path.argtypes = [vp]
+        lib.mcce_route_trace_static_limit.restype = C.c_size_t
+        lib.mcce_route_trace_static.argtypes = [C.POINTER(Config), i32, vp, vp, vp, vp, vp, vp, C.POINTER(Stats), vp]
         lib.mcce_profile.argtypes = [vp, C.c_int]
         lib.mcce_profile_read.argtypes = [vp, vp, vp, C.c_int]
         lib.mcce_gen_normal.argtypes = [vp, i32, u64, u64, u32, u32, u32, f32, vp]
@@ -266,3 +269,23 @@ def gen_philox_words(n_blocks: int, seed: int, tensor_id: int, t: int, start_blo
     out = torch.empty((n_blocks, 4), dtype=torch.int32, device=device)
     _check(load().mcce_gen_philox_words(_ptr(out), start_block, n_blocks, seed, tensor_id, t, _stream()))
     return out
+
+
+def route_trace_static(*, L, E, K, J, C_cap, S, lam, logits=None, hidden=None, Wr=None, fixed_delta=None,
+                       delta_mode=DELTA_RUNNING, renorm=1, want_totals=True):
+    """Routing over a whole trace from empty caches through the entry point that allocates nothing inside
+    the library (its cache state lives in a fixed array of the library image).  Output tensors are the
+    caller's; here they are torch tensors for convenience.  Returns sel_idx, sel_w[, totals]."""
+    src = logits if logits is not None else hidden
+    n_steps = src.shape[0]
+    d = hidden.shape[-1] if hidden is not None else 8
+    dtype = BF16 if (hidden is not None and hidden.dtype == torch.bfloat16) else F32
+    cfg = Config(L, E, K, J, 0, d, 8, C_cap, S, lam, delta_mode, renorm, dtype, dtype, 0, src.device.index or 0)
+    sel = torch.empty((n_steps, L, S, K), dtype=torch.int32, device=src.device)
+    w = torch.empty((n_steps, L, S, K), dtype=torch.float32, device=src.device)
+    totals = Stats()
+    with torch.cuda.device(src.device):
+        _check(load().mcce_route_trace_static(C.byref(cfg), n_steps, _ptr(hidden), _ptr(Wr), _ptr(logits),
+                                              _ptr(fixed_delta), _ptr(sel), _ptr(w),
+                                              C.byref(totals) if want_totals else None, _stream()))
+    return (sel, w, totals.as_tuple()) if want_totals else (sel, w)

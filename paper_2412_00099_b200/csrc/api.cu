@@ -448,6 +448,9 @@ extern "C" const char* mcce_strerror(int code) {
     case MCCE_ESTATE: return "weights not set, or a 32-bit recency counter would overflow (call mcce_reset)";
     case MCCE_ECUDA: return "CUDA call failed (see mcce_last_cuda_error)";
     case MCCE_ETIMEOUT: return "a bounded wait inside a kernel gave up";
+    case MCCE_ELIMIT:
+      return "the cache state of this configuration exceeds the fixed 4 MiB array of mcce_route_trace_static "
+             "(use mcce_create with a workspace instead)";
     default: return "unknown error";
   }
 }
