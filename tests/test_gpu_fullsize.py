@@ -1,0 +1,119 @@
+"""Parity at full size, in the configuration the benchmark times: the Qwen1.5-MoE-A2.7B-shaped workload
+(24 layers x 256 streams, 60+4 experts, bf16, tensor-core FFN path, one route + forward per token).
+
+The library's inputs are generated on the device; the oracle's inputs for the sampled (layer, stream)
+pairs are regenerated on the host from the same seeded definition (the two generators agree bit for bit,
+which is re-checked here on the sampled expert matrices).  Sampled outputs are compared one by one; the
+rest is checked through properties that hold at any size."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2412_00099_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+T_STEPS = 5
+SAMPLES = [(0, 0), (3, 17), (11, 128), (23, 255), (7, 64), (16, 201)]   # (layer, stream)
+FFN_SAMPLES = 4                                                        # pairs whose FFN output is recomputed
+
+
+def bits(t: torch.Tensor) -> np.ndarray:
+    return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+@pytest.mark.parametrize("wl", [synth.QWEN])
+def test_full_size_sampled_parity(wl):
+    from oracle import oracle as orc
+    from paper_2412_00099_b200 import binding as mb
+    import helpers as H
+
+    dev = torch.device("cuda")
+    bf = torch.bfloat16
+    eng = mb.engine_for(wl)
+    assert eng.uses_tensor_path()
+    Wr = mb.gen_normal(torch.empty((wl.L, wl.E, wl.d), dtype=torch.float32, device=dev), wl.seed, synth.T_ROUTER,
+                       std=wl.weight_std)
+    up, dn = (wl.L, wl.E, wl.I, wl.d), (wl.L, wl.E, wl.d, wl.I)
+    sup, sdn = (wl.L, wl.n_shared, wl.I, wl.d), (wl.L, wl.n_shared, wl.d, wl.I)
+    W = {"Wg": (synth.T_WG, up), "Wu": (synth.T_WU, up), "Wd": (synth.T_WD, dn), "shWg": (synth.T_SH_WG, sup),
+         "shWu": (synth.T_SH_WU, sup), "shWd": (synth.T_SH_WD, sdn)}
+    Wt = {k: mb.gen_normal(torch.empty(shp, dtype=bf, device=dev), wl.seed, tid, std=wl.weight_std)
+          for k, (tid, shp) in W.items()}
+    eng.set_router(Wr)
+    eng.set_experts(**Wt)
+    assert np.array_equal(Wr.cpu().numpy(), wl.router())          # router: device generator == host generator
+
+    # the oracle follows the sampled pairs only: one "layer" per sample, one stream each
+    n = len(SAMPLES)
+    Wr_s = np.ascontiguousarray(wl.router()[[l for l, _ in SAMPLES]])
+    o = orc.Oracle(orc.OracleConfig(n, wl.E, wl.K, wl.J, wl.n_shared, wl.d, wl.I, wl.C, 1, wl.lam, 0, 1, 1))
+    host_x = wl.hidden_trace(T_STEPS, rows=SAMPLES)
+
+    state = torch.empty(wl.L * wl.S * wl.d, dtype=torch.float32, device=dev)
+    x = torch.empty((wl.L, wl.S, wl.d), dtype=bf, device=dev)
+    near = 0
+    for t in range(T_STEPS):
+        mb.gen_hidden_step(state, x, wl.seed, t, wl.rho, wl.topic_offset)
+        sel, w, z = eng.route_step(hidden=x, want_logits=True)
+        y = eng.moe_forward(x, sel[0], w[0])
+        sel_h, w_h, z_h, y_h = sel[0].cpu().numpy(), w[0].cpu().numpy(), z[0].cpu().numpy(), y.cpu().numpy()
+
+        # ---- properties at full size ----------------------------------------------------------------
+        assert np.isfinite(y_h).all()
+        assert (np.sort(sel_h, -1)[..., 1:] != np.sort(sel_h, -1)[..., :-1]).all()       # K distinct experts
+        assert sel_h.min() >= 0 and sel_h.max() < wl.E
+        assert np.allclose(w_h.sum(-1), 1.0, atol=1e-5)
+        topj = np.argsort(-z_h, -1, kind="stable")[..., :wl.J]
+        assert all((topj[..., j:j + 1] == sel_h).any(-1).all() for j in range(wl.J))     # top-J always selected
+        offsets, perm = eng.grouping()
+        for l in range(0, wl.L, 5):
+            flat = sel_h[l].reshape(-1)
+            assert np.array_equal(offsets[l], np.concatenate([[0], np.cumsum(np.bincount(flat, minlength=wl.E))]))
+            assert np.array_equal(perm[l], np.argsort(flat, kind="stable"))
+
+        # ---- sampled pairs against the oracle --------------------------------------------------------
+        xs = next(host_x)                                              # [n, d] bf16 bits from the host generator
+        for i, (l, s) in enumerate(SAMPLES):
+            assert np.array_equal(bits(x[l, s]), xs[i])                # same inputs on both sides
+        z_g = np.stack([z_h[l, s] for l, s in SAMPLES])[:, None, :]
+        z_own = o.logits(Wr_s, xs.reshape(n, 1, wl.d))
+        assert (np.abs(z_g - z_own) <= H.LOGIT_RTOL * np.maximum(1.0, np.abs(z_own))).all()
+        snap = o.snapshot()
+        sel_own, _, margin, _ = o.route(z_own, want_margin=True)
+        o.restore(snap)
+        osel, ow = o.route(z_g)
+        for i, (l, s) in enumerate(SAMPLES):
+            assert np.array_equal(sel_h[l, s], osel[i, 0])
+            assert np.allclose(w_h[l, s], ow[i, 0], rtol=1e-5, atol=1e-7)
+            if not np.array_equal(sel_own[i, 0], osel[i, 0]):
+                assert margin[i, 0] < H.NEAR_TIE
+                near += 1
+
+        if t == T_STEPS - 1:                                           # FFN outputs of a few pairs, recomputed
+            for i, (l, s) in enumerate(SAMPLES[:FFN_SAMPLES]):
+                acc = np.zeros(wl.d, np.float64)
+                for k in range(wl.K):
+                    e = int(osel[i, 0, k])
+                    mats = [wl.expert_matrix(tid, l, e) for tid in (synth.T_WG, synth.T_WU, synth.T_WD)]
+                    if k == 0:                                         # device weights == host weights
+                        assert np.array_equal(bits(Wt["Wg"][l, e]), mats[0])
+                        assert np.array_equal(bits(Wt["Wd"][l, e]), mats[2])
+                    acc += float(ow[i, 0, k]) * orc.expert_ffn(xs[i], *mats, 1)
+                for q in range(wl.n_shared):
+                    mats = [wl.expert_matrix(tid, l, q) for tid in (synth.T_SH_WG, synth.T_SH_WU, synth.T_SH_WD)]
+                    acc += orc.expert_ffn(xs[i], *mats, 1)
+                err = H.ffn_close(y_h[l, s], acc.astype(np.float32))
+                print("full-size FFN sample (l=%d, s=%d): max abs err %.2e" % (l, s, err[0]))
+
+    # cache state and counters of the sampled pairs
+    order, ever, dsum, cnt = eng.cache_state()
+    o_order = o.order()
+    for i, (l, s) in enumerate(SAMPLES):
+        assert np.array_equal(order[l, s], o_order[i, 0])
+        assert np.array_equal(ever[l, s], o.ever[i, 0])
+        assert dsum[l, s].view(np.uint32) == o.sum_range[i, 0].view(np.uint32)
+    total, per_layer = eng.cache_stats()
+    assert total[0] == T_STEPS * wl.L * wl.S and total[1] == total[0] * wl.K
+    assert 0 < total[3] <= total[2] <= total[1]
+    print("full size: %d sampled steps, %d near ties, miss rate %.3f" % (T_STEPS * n, near, total[2] / total[1]))
