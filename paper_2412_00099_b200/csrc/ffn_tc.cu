@@ -158,23 +158,33 @@ __device__ __forceinline__ uint32_t instr_desc(uint32_t n) {
 }
 
 // ---- the list of work items ----------------------------------------------------------------------------
+// Per layer: one item per (routed expert, 128-row tile), covering all of the expert's tokens (in passes
+// of kNMax), then one item per (shared expert, 128-row tile, 128-token pass).  A shared expert sees
+// every stream, so its passes are separate, adjacent items: neighbouring CTAs run them at the same
+// time and the second read of the weight tile is served by L2 instead of HBM.
 struct Item {
-  int m;          // tokens of the group
+  int m;          // tokens this item covers
   int wrow;       // first row of the 128-row weight tile in the weight tensor map
   int xrow;       // first token row in the activation tensor map
-  size_t orow;    // first row of the group in H / O
+  size_t orow;    // first row in H / O
   int col0;       // first output column (= weight row inside the expert) of this tile
   bool shared;
 };
 
+__host__ __device__ __forceinline__ int items_per_layer(int E, int n_sh, int S, int RT) {
+  return E * RT + n_sh * RT * ((S + kNMax - 1) / kNMax);
+}
+
 template <bool UP>
 __device__ __forceinline__ Item decode(const TcArgs& a, int w) {
   const int rows = UP ? a.I : a.d;
-  const int RT = rows / kTileM, G = a.E + a.n_sh, P = a.S * a.K;
-  const int rt = w % RT, g = (w / RT) % G, l = w / (RT * G);
+  const int RT = rows / kTileM, P = a.S * a.K, NC = (a.S + kNMax - 1) / kNMax;
+  const int per_layer = items_per_layer(a.E, a.n_sh, a.S, RT);
+  const int l = w / per_layer, wl = w % per_layer;
   Item it;
-  it.col0 = rt * kTileM;
-  if (g < a.E) {
+  if (wl < a.E * RT) {
+    const int g = wl / RT;
+    it.col0 = (wl % RT) * kTileM;
     const int o0 = __ldg(a.offsets + (size_t)l * (a.E + 1) + g);
     it.m = __ldg(a.offsets + (size_t)l * (a.E + 1) + g + 1) - o0;
     it.shared = false;
@@ -182,12 +192,14 @@ __device__ __forceinline__ Item decode(const TcArgs& a, int w) {
     it.xrow = l * P + o0;
     it.orow = (size_t)it.xrow;
   } else {
-    const int q = g - a.E;
-    it.m = a.S;
+    const int idx = wl - a.E * RT;
+    const int c = idx % NC, rt = (idx / NC) % RT, q = idx / (NC * RT);
+    it.col0 = rt * kTileM;
+    it.m = min(kNMax, a.S - c * kNMax);
     it.shared = true;
     it.wrow = (l * a.n_sh + q) * rows + it.col0;
-    it.orow = (size_t)a.L * P + (size_t)(l * a.n_sh + q) * a.S;
-    it.xrow = UP ? l * a.S : (int)it.orow;   // up: rows of the hidden tensor; down: rows of H
+    it.orow = (size_t)a.L * P + (size_t)(l * a.n_sh + q) * a.S + c * kNMax;
+    it.xrow = UP ? l * a.S + c * kNMax : (int)it.orow;   // up: rows of the hidden tensor; down: rows of H
   }
   return it;
 }
@@ -404,7 +416,7 @@ cudaError_t launch(const TcMaps& maps, const FfnParams& p, uint32_t* err, cudaSt
   }
   TcArgs a;
   a.L = p.L, a.S = p.S, a.E = p.E, a.K = p.K, a.n_sh = p.n_sh, a.d = p.d, a.I = p.I;
-  a.n_items = p.L * (p.E + p.n_sh) * ((UP ? p.I : p.d) / kTileM);
+  a.n_items = p.L * items_per_layer(p.E, p.n_sh, p.S, (UP ? p.I : p.d) / kTileM);
   a.offsets = p.offsets, a.H = (__nv_bfloat16*)p.H, a.O = p.O, a.err = err;
   const int grid = a.n_items < sms ? a.n_items : sms;
   ffn_tc_kernel<UP><<<grid, kThreads, Cfg<UP>::kSmemBytes, st>>>(maps, a);
