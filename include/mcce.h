@@ -160,13 +160,14 @@ int mcce_gen_philox_words(uint32_t* out, uint64_t start_block, uint64_t n_blocks
  * recorded events and returns, per kernel kind, the summed milliseconds and the number of launches
  * (HOST arrays of MCCE_N_KERNELS entries), clearing the sums if reset != 0. */
 enum {
-  MCCE_K_ROUTE = 0,    /* fused route kernel                         */
+  MCCE_K_ROUTE = 0,    /* fused route kernel (with bf16 hidden states: its tail, on the logits of MCCE_K_ROUTE_GEMM) */
   MCCE_K_GROUP = 1,    /* histogram + scan + scatter                 */
   MCCE_K_GATHER = 2,   /* activation rows into expert order          */
   MCCE_K_FFN_UP = 3,   /* H = silu(X Wg^T) * (X Wu^T), all groups    */
   MCCE_K_FFN_DOWN = 4, /* O = H Wd^T, all groups                     */
   MCCE_K_COMBINE = 5,  /* weighted sum over slots + shared experts   */
-  MCCE_N_KERNELS = 6
+  MCCE_K_ROUTE_GEMM = 6, /* router logits on the tensor cores (bf16 hidden states) */
+  MCCE_N_KERNELS = 7
 };
 int mcce_profile(mcce_ctx* ctx, int enable);
 int mcce_profile_read(mcce_ctx* ctx, double* ms /*HOST*/, int64_t* launches /*HOST*/, int reset);

@@ -215,7 +215,7 @@ class Engine:
         _check(self.lib.mcce_get_cache_state(self.ctx, _ptr(order), _ptr(ever), _ptr(dsum), C.byref(cnt)), self.ctx)
         return order, ever, dsum, cnt.value
 
-    KERNELS = ("route", "group", "gather", "ffn_up", "ffn_down", "combine")
+    KERNELS = ("route", "group", "gather", "ffn_up", "ffn_down", "combine", "route_gemm")
 
     def uses_tensor_path(self) -> bool:
         return self.lib.mcce_uses_tensor_path(self.ctx) == 1

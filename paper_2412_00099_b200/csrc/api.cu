@@ -35,6 +35,10 @@ struct mcce_ctx {
   int last_cuda;
   int use_tc;
   TcPlan tc;
+  int use_tc_router;
+  RouterGemmPlan rg;
+  void* wr_terms;
+  float* z_buf;
   // optional per-kernel timing: event pairs recorded around each launch, summed by mcce_profile_read
   int profiling;
   int n_pairs;
@@ -69,7 +73,7 @@ bool valid(const mcce_config* c) {
 
 struct Layout {
   size_t stamp, ever, sum_range, miss, cold, err, stats, offsets, perm, inv, Xg, H, O, st_hidden, st_sel, st_w, st_y,
-      total;
+      wr_terms, z_buf, total;
 };
 
 Layout layout_of(const mcce_config& c) {
@@ -100,6 +104,9 @@ Layout layout_of(const mcce_config& c) {
   o.st_sel = take(L * S * K * 4);
   o.st_w = take(L * S * K * 4);
   o.st_y = take(L * S * d * 4);
+  const bool rg = router_gemm_applicable(c);
+  o.wr_terms = take(rg ? 3 * L * E * d * 2 : 0);
+  o.z_buf = take(rg ? (size_t)router_gemm_steps_max() * L * S * E * 4 : 0);
   o.total = p;
   return o;
 }
@@ -190,6 +197,8 @@ extern "C" int mcce_create(const mcce_config* cfg, void* workspace, size_t works
   ctx->stage_hidden = w + lo.st_hidden, ctx->stage_sel = (int32_t*)(w + lo.st_sel);
   ctx->stage_w = (float*)(w + lo.st_w), ctx->stage_y = (float*)(w + lo.st_y);
   ctx->use_tc = cfg->ffn_impl != MCCE_FFN_SIMT && tc_applicable(*cfg);
+  ctx->use_tc_router = router_gemm_applicable(*cfg);
+  ctx->wr_terms = w + lo.wr_terms, ctx->z_buf = (float*)(w + lo.z_buf);
   cudaError_t e = cudaSetDevice(cfg->device);
   // state arrays and the activation buffers start at zero (the slack rows must hold finite values)
   if (e == cudaSuccess) e = cudaMemset(w, 0, lo.O);
@@ -219,6 +228,12 @@ extern "C" int mcce_set_router(mcce_ctx* ctx, const float* Wr, const float* fixe
   if ((uintptr_t)Wr % 16) return MCCE_EINVAL;
   ctx->Wr = Wr;
   ctx->fixed_delta = fixed_delta;
+  if (ctx->use_tc_router) {
+    CK(cudaSetDevice(ctx->cfg.device));
+    const int rc = router_gemm_plan(ctx->cfg, Wr, ctx->wr_terms, &ctx->rg, 0);
+    if (rc != MCCE_OK) return rc;
+    CK(cudaDeviceSynchronize());
+  }
   return MCCE_OK;
 }
 
@@ -288,13 +303,33 @@ extern "C" int mcce_route_step(mcce_ctx* ctx, int32_t n_steps, const void* hidde
   if (last_key >= 0xffffffffull || ctx->delta_cnt + n_steps >= 0xffffffffull) return MCCE_ESTATE;
   RouteParams p;
   p.L = c.n_layers, p.S = c.n_streams, p.E = c.n_experts, p.K = c.top_k, p.J = c.top_j, p.C = c.cache_capacity;
-  p.d = c.d_model, p.n_steps = n_steps, p.lambda = c.lambda, p.delta_mode = c.delta_mode, p.renorm = c.renorm;
+  p.d = c.d_model, p.lambda = c.lambda, p.delta_mode = c.delta_mode, p.renorm = c.renorm;
   p.hidden_bf16 = c.hidden_dtype == MCCE_BF16;
-  p.hidden = hidden, p.logits_in = logits_in, p.Wr = ctx->Wr, p.fixed_delta = ctx->fixed_delta;
+  p.Wr = ctx->Wr, p.fixed_delta = ctx->fixed_delta;
   p.stamp = ctx->stamp, p.ever = ctx->ever, p.sum_range = ctx->sum_range, p.miss = ctx->miss, p.cold = ctx->cold;
-  p.sel_idx = sel_idx, p.sel_w = sel_w, p.logits_out = logits_out;
-  p.tok0 = (uint32_t)ctx->tok, p.cnt0 = (uint32_t)ctx->delta_cnt;
-  TIMED(MCCE_K_ROUTE, (cudaStream_t)cuda_stream, launch_route(p, (cudaStream_t)cuda_stream));
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  if (hidden && ctx->use_tc_router && ctx->rg.ready) {
+    // logits by the tensor-core GEMM, a few tokens at a time, then the fused tail on those logits
+    const size_t LS = (size_t)c.n_layers * c.n_streams, esz = 2;
+    for (int t0 = 0; t0 < n_steps; t0 += router_gemm_steps_max()) {
+      const int nt = n_steps - t0 < router_gemm_steps_max() ? n_steps - t0 : router_gemm_steps_max();
+      const char* h = (const char*)hidden + (size_t)t0 * LS * c.d_model * esz;
+      TIMED(MCCE_K_ROUTE_GEMM, st, router_gemm_launch(ctx->rg, c, h, nt, ctx->z_buf, ctx->err, st));
+      p.n_steps = nt, p.hidden = nullptr, p.logits_in = ctx->z_buf;
+      p.sel_idx = sel_idx + (size_t)t0 * LS * c.top_k, p.sel_w = sel_w + (size_t)t0 * LS * c.top_k;
+      p.logits_out = nullptr;
+      p.tok0 = (uint32_t)(ctx->tok + t0), p.cnt0 = (uint32_t)(ctx->delta_cnt + t0);
+      TIMED(MCCE_K_ROUTE, st, launch_route(p, st));
+      if (logits_out)
+        CK(cudaMemcpyAsync(logits_out + (size_t)t0 * LS * c.n_experts, ctx->z_buf, (size_t)nt * LS * c.n_experts * 4,
+                           cudaMemcpyDeviceToDevice, st));
+    }
+  } else {
+    p.n_steps = n_steps, p.hidden = hidden, p.logits_in = logits_in;
+    p.sel_idx = sel_idx, p.sel_w = sel_w, p.logits_out = logits_out;
+    p.tok0 = (uint32_t)ctx->tok, p.cnt0 = (uint32_t)ctx->delta_cnt;
+    TIMED(MCCE_K_ROUTE, st, launch_route(p, st));
+  }
   ctx->tok += n_steps;
   ctx->steps_since_reset += n_steps;
   if (c.delta_mode == MCCE_DELTA_RUNNING) ctx->delta_cnt += n_steps;

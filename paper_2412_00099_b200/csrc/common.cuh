@@ -1,5 +1,6 @@
 // Internal declarations shared by the translation units of libmcce.so.
 #pragma once
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -58,6 +59,19 @@ struct FfnParams {
   float* O;                // [rows, d]    expert outputs
   float* y;                // [L,S,d]
 };
+
+// Router logits on the tensor cores (route_gemm.cu).  Plain data: lives inside the zero-initialised context.
+struct RouterGemmPlan {
+  alignas(64) CUtensorMap w, x;
+  const void* hidden_ptr;
+  uint64_t hidden_rows;
+  int ready;
+};
+bool router_gemm_applicable(const mcce_config& c);
+int router_gemm_steps_max();
+int router_gemm_plan(const mcce_config& c, const float* Wr, void* terms, RouterGemmPlan* plan, cudaStream_t st);
+cudaError_t router_gemm_launch(RouterGemmPlan& plan, const mcce_config& c, const void* hidden, int n_steps, float* Z,
+                               uint32_t* err, cudaStream_t st);
 
 cudaError_t launch_route(const RouteParams& p, cudaStream_t st);
 cudaError_t launch_group(const GroupParams& p, cudaStream_t st);

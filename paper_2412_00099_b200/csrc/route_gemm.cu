@@ -1,0 +1,305 @@
+// Router logits of Eq. 3 on the tensor cores: Z[(t,l,s), e] = sum_j W_r[l][e][j] x[(t,l,s)][j].
+//
+// Every stream of a layer shares the layer's router matrix, so the S GEMVs of a layer are one GEMM.  The
+// routing decision needs near-fp32 logits (ties are resolved at 1e-4), while tcgen05 multiplies bf16:
+// the fp32 router is therefore split once, at set-up, into three bf16 terms W = hi + mid + lo (each the
+// bf16 rounding of what the previous terms left), and the kernel accumulates the three products in the
+// fp32 TMEM accumulators.  The hidden states are bf16 already, so every product is exact.
+//
+// Accuracy: the tensor core's fp32 accumulate truncates, which over the 3*d/16 accumulate steps of one
+// logit would add up to a bias of about 1e-5 relative.  The kernel therefore (i) keeps the large hi
+// products and the small mid/lo products in separate accumulators, and (ii) ends an accumulation phase
+// every kPhaseSlabs K-slabs: the epilogue warps add each phase's two partial sums into fp32 registers
+// with round-to-nearest adds while the MMA warp continues in the other TMEM buffer.
+//
+// Layout of the work: swapped GEMM as in the expert kernels -- router rows (experts) are MMA M (tiles of
+// 128, rows past E zero-filled by TMA at no memory cost), a block of streams is MMA N, the hidden
+// dimension is K in 64-column slabs.  Persistent CTAs walk (token, layer, expert tile, stream block)
+// items: warp 0 TMA producer, warp 1 MMA issuer, warps 2-5 epilogue (TMEM -> fp32 logits in HBM), with
+// bounded mbarrier waits throughout.  The fused routing tail then runs on these logits.
+#include "common.cuh"
+#include "tc_common.cuh"
+
+namespace mcce {
+
+using namespace tc;
+
+namespace {
+
+constexpr int kTileM = 128, kTileK = 64, kNSMax = 64, kXBox = 16, kThreads = 192, kStages = 4;
+constexpr uint32_t kABytes = kTileM * kTileK * 2;          // one bf16 term of the router tile: 16 KB
+constexpr uint32_t kBBytes = kNSMax * kTileK * 2;          // stream rows: 8 KB
+constexpr uint32_t kStageBytes = 3 * kABytes + kBBytes;    // 56 KB
+constexpr int kAccCols = 2 * kNSMax, kTmemCols = 2 * kAccCols; // per buffer: hi + mid/lo partial sums; 2 buffers
+constexpr int kPhaseSlabs = 4;                             // K-slabs (of 64) per accumulation phase
+constexpr size_t kSmemBytes = (size_t)kStages * kStageBytes + 1024 + 256;
+
+struct GemmArgs {
+  int L, S, E, d, n_steps, NS;
+  int n_items;
+  float* Z;        // [n_steps, L, S, E]
+  uint32_t* err;
+};
+struct GemmMaps {
+  CUtensorMap w;   // 3-D: [3*L][E][d] bf16 terms (term-major), box 1 x 128 x 64
+  CUtensorMap x;   // 2-D: [n_steps*L*S][d] hidden rows, box 16 x 64
+};
+
+struct GItem {
+  int l, mt, s0, row0;  // layer, expert tile, first stream, first hidden row (t*L + l)*S + s0
+};
+
+__device__ __forceinline__ GItem decode(const GemmArgs& a, int w) {
+  const int SB = (a.S + a.NS - 1) / a.NS, MT = (a.E + kTileM - 1) / kTileM;
+  GItem it;
+  const int sb = w % SB;
+  it.mt = (w / SB) % MT;
+  it.l = (w / (SB * MT)) % a.L;
+  const int t = w / (SB * MT * a.L);
+  it.s0 = sb * a.NS;
+  it.row0 = (t * a.L + it.l) * a.S + it.s0;
+  return it;
+}
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z)
+      : "memory");
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+router_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs a) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_al = smem_raw + (smem_base - smem_u32(smem_raw));
+  uint64_t* bars = (uint64_t*)(smem_al + (size_t)kStages * kStageBytes);
+  const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * kStages;
+  const uint32_t bar_tfull = bar_empty + 8 * kStages, bar_tempty = bar_tfull + 16;
+  uint32_t* tmem_slot = (uint32_t*)(bars + 2 * kStages + 4);
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int KT = a.d / kTileK;
+  const uint32_t n = (uint32_t)a.NS;   // MMA N: multiple of 16
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(bar_full + 8 * s, 1);
+      mbar_init(bar_empty + 8 * s, 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(bar_tfull + 8 * b, 1);
+      mbar_init(bar_tempty + 8 * b, 4);
+    }
+    *abort_flag = 0u;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      uint32_t stage = 0, phase = 0;
+      bool alive = true;
+      const uint32_t tx = 3 * kABytes + n * kTileK * 2;
+      for (int w = blockIdx.x; w < a.n_items && alive; w += gridDim.x) {
+        const GItem it = decode(a, w);
+        for (int kt = 0; kt < KT; ++kt) {
+          if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, a.err, 11u)) {
+            alive = false;
+            break;
+          }
+          const uint32_t sa = smem_base + stage * kStageBytes, full = bar_full + 8 * stage;
+          mbar_expect_tx(full, tx);
+#pragma unroll
+          for (int p = 0; p < 3; ++p)
+            tma_load_3d(sa + p * kABytes, &maps.w, kt * kTileK, it.mt * kTileM, p * a.L + it.l, full);
+          const uint32_t sb = sa + 3 * kABytes;
+          for (int j = 0; j < a.NS; j += kXBox)
+            tma_load_2d(sb + j * kTileK * 2, &maps.x, kt * kTileK, it.row0 + j, full);
+          if (++stage == kStages) stage = 0, phase ^= 1u;
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      uint32_t stage = 0, phase = 0, acc_iter = 0;
+      bool alive = true;
+      const uint32_t idesc = instr_desc(n);
+      for (int w = blockIdx.x; w < a.n_items && alive; w += gridDim.x) {
+        for (int k0 = 0; k0 < KT && alive; k0 += kPhaseSlabs, ++acc_iter) {
+          const uint32_t buf = acc_iter & 1u, acc_phase = (acc_iter >> 1) & 1u;
+          if (!mbar_wait(bar_tempty + 8 * buf, acc_phase ^ 1u, abort_flag, a.err, 12u)) {
+            alive = false;
+            break;
+          }
+          tc_fence_after();
+          const uint32_t d_hi = tmem_base + buf * kAccCols, d_lo = d_hi + kNSMax;
+          const int k1 = min(KT, k0 + kPhaseSlabs);
+          for (int kt = k0; kt < k1; ++kt) {
+            if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag, a.err, 13u)) {
+              alive = false;
+              break;
+            }
+            tc_fence_after();
+            const uint32_t sa = smem_base + stage * kStageBytes, sb = sa + 3 * kABytes;
+#pragma unroll
+            for (int k = 0; k < kTileK / 16; ++k) {
+              const uint64_t bd = smem_desc(sb + k * 32);
+              const uint32_t first = (kt == k0 && k == 0) ? 0u : 1u;
+              umma_bf16(d_hi, smem_desc(sa + k * 32), bd, idesc, first);
+              umma_bf16(d_lo, smem_desc(sa + kABytes + k * 32), bd, idesc, first);
+              umma_bf16(d_lo, smem_desc(sa + 2 * kABytes + k * 32), bd, idesc, 1u);
+            }
+            umma_commit(bar_empty + 8 * stage);
+            if (++stage == kStages) stage = 0, phase ^= 1u;
+          }
+          if (alive) umma_commit(bar_tfull + 8 * buf);
+        }
+      }
+    }
+  } else {
+    const int quad = warp & 3;
+    const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+    uint32_t acc_iter = 0;
+    bool alive = true;
+    for (int w = blockIdx.x; w < a.n_items && alive; w += gridDim.x) {
+      const GItem it = decode(a, w);
+      const int e = it.mt * kTileM + quad * 32 + lane;
+      float zacc[kNSMax];
+#pragma unroll
+      for (int j = 0; j < kNSMax; ++j) zacc[j] = 0.f;
+      for (int k0 = 0; k0 < KT && alive; k0 += kPhaseSlabs, ++acc_iter) {
+        const uint32_t buf = acc_iter & 1u, acc_phase = (acc_iter >> 1) & 1u;
+        if (!mbar_wait(bar_tfull + 8 * buf, acc_phase, abort_flag, a.err, 14u)) {
+          alive = false;
+          break;
+        }
+        tc_fence_after();
+        const uint32_t t0 = tmem_base + lane_addr + buf * kAccCols;
+#pragma unroll
+        for (int n0 = 0; n0 < kNSMax; n0 += 16) {
+          if (n0 < a.NS) {
+            float hi[16], lo[16];
+            tmem_ld16(t0 + n0, hi);
+            tmem_ld16(t0 + kNSMax + n0, lo);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 16; ++j) zacc[n0 + j] = __fadd_rn(zacc[n0 + j], __fadd_rn(hi[j], lo[j]));
+          }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);
+      }
+      if (alive && e < a.E) {
+#pragma unroll
+        for (int j = 0; j < kNSMax; ++j)
+          if (j < a.NS && it.s0 + j < a.S) a.Z[(size_t)(it.row0 + j) * a.E + e] = zacc[j];
+      }
+    }
+  }
+
+  __syncwarp();
+  if (*abort_flag) {
+    const unsigned long long t0 = global_ns();
+    while (global_ns() - t0 < 200000ull) __nanosleep(1000);
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
+}
+
+// W (fp32) -> hi, mid, lo (bf16): each term is the bf16 rounding of what the earlier terms left over.
+__global__ void split_router_kernel(const float* W, __nv_bfloat16* out, size_t n) {
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+    const float w = W[i];
+    const __nv_bfloat16 hi = __float2bfloat16_rn(w);
+    const float r1 = __fsub_rn(w, __bfloat162float(hi));
+    const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
+    const float r2 = __fsub_rn(r1, __bfloat162float(mid));
+    out[i] = hi;
+    out[n + i] = mid;
+    out[2 * n + i] = __float2bfloat16_rn(r2);
+  }
+}
+
+}  // namespace
+
+bool router_gemm_applicable(const mcce_config& c) { return c.hidden_dtype == MCCE_BF16 && c.d_model % kTileK == 0; }
+
+int router_gemm_steps_max() { return 8; }
+
+// Splits the router into its bf16 terms (device buffer `terms`, 3*L*E*d bf16) and describes them to TMA.
+int router_gemm_plan(const mcce_config& c, const float* Wr, void* terms, RouterGemmPlan* plan, cudaStream_t st) {
+  const size_t n = (size_t)c.n_layers * c.n_experts * c.d_model;
+  split_router_kernel<<<(unsigned)((n + 255) / 256 > 4096 ? 4096 : (n + 255) / 256), 256, 0, st>>>(
+      Wr, (__nv_bfloat16*)terms, n);
+  if (cudaGetLastError() != cudaSuccess) return MCCE_ECUDA;
+  EncodeFn fn = encode_fn();
+  if (!fn) return MCCE_ECUDA;
+  const cuuint64_t dims[3] = {(cuuint64_t)c.d_model, (cuuint64_t)c.n_experts, (cuuint64_t)3 * c.n_layers};
+  const cuuint64_t strides[2] = {(cuuint64_t)c.d_model * 2, (cuuint64_t)c.d_model * 2 * c.n_experts};
+  const cuuint32_t box[3] = {(cuuint32_t)kTileK, (cuuint32_t)kTileM, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  if (fn(&plan->w, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, terms, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+         CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return MCCE_ECUDA;
+  plan->hidden_ptr = nullptr;
+  plan->hidden_rows = 0;
+  plan->ready = 1;
+  return MCCE_OK;
+}
+
+cudaError_t router_gemm_launch(RouterGemmPlan& plan, const mcce_config& c, const void* hidden, int n_steps, float* Z,
+                               uint32_t* err, cudaStream_t st) {
+  static int sms = 0;
+  if (!sms) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    cudaError_t e = cudaFuncSetAttribute(router_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)kSmemBytes);
+    if (e != cudaSuccess) {
+      sms = 0;
+      return e;
+    }
+  }
+  const uint64_t rows = (uint64_t)n_steps * c.n_layers * c.n_streams;
+  if (plan.hidden_ptr != hidden || plan.hidden_rows != rows) {
+    EncodeFn fn = encode_fn();
+    const cuuint64_t dims[2] = {(cuuint64_t)c.d_model, rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)c.d_model * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kTileK, (cuuint32_t)kXBox};
+    const cuuint32_t estr[2] = {1, 1};
+    if (!fn || fn(&plan.x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(hidden), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return cudaErrorInvalidValue;
+    plan.hidden_ptr = hidden;
+    plan.hidden_rows = rows;
+  }
+  GemmArgs a;
+  a.L = c.n_layers, a.S = c.n_streams, a.E = c.n_experts, a.d = c.d_model, a.n_steps = n_steps;
+  // streams per tile: as many as 64, fewer when that would leave most SMs without a tile
+  int ns = c.n_streams >= kNSMax ? kNSMax : (c.n_streams + 15) & ~15;
+  const int mt = (c.n_experts + kTileM - 1) / kTileM;
+  while (ns > 16 && n_steps * c.n_layers * mt * ((c.n_streams + ns - 1) / ns) < sms / 2) ns /= 2;
+  ns = (ns + 15) & ~15;
+  a.NS = ns;
+  a.n_items = n_steps * c.n_layers * mt * ((c.n_streams + ns - 1) / ns);
+  a.Z = Z, a.err = err;
+  GemmMaps m;
+  m.w = plan.w, m.x = plan.x;
+  const int grid = a.n_items < sms ? a.n_items : sms;
+  router_gemm_kernel<<<grid, kThreads, kSmemBytes, st>>>(m, a);
+  return cudaGetLastError();
+}
+
+}  // namespace mcce
