@@ -314,18 +314,17 @@ extern "C" int mcce_route_step(mcce_ctx* ctx, int32_t n_steps, const void* hidde
     for (int t0 = 0; t0 < n_steps; t0 += router_gemm_steps_max()) {
       const int nt = n_steps - t0 < router_gemm_steps_max() ? n_steps - t0 : router_gemm_steps_max();
       const char* h = (const char*)hidden + (size_t)t0 * LS * c.d_model * esz;
-      TIMED(MCCE_K_ROUTE_GEMM, st, router_gemm_launch(ctx->rg, c, h, nt, ctx->z_buf, ctx->err, st));
+      int ks = 1;
+      TIMED(MCCE_K_ROUTE_GEMM, st, router_gemm_launch(ctx->rg, c, h, nt, ctx->z_buf, &ks, ctx->err, st));
       p.n_steps = nt, p.hidden = nullptr, p.logits_in = ctx->z_buf;
+      p.n_partials = ks, p.partial_stride = (size_t)nt * LS * c.n_experts;
       p.sel_idx = sel_idx + (size_t)t0 * LS * c.top_k, p.sel_w = sel_w + (size_t)t0 * LS * c.top_k;
-      p.logits_out = nullptr;
+      p.logits_out = logits_out ? logits_out + (size_t)t0 * LS * c.n_experts : nullptr;
       p.tok0 = (uint32_t)(ctx->tok + t0), p.cnt0 = (uint32_t)(ctx->delta_cnt + t0);
       TIMED(MCCE_K_ROUTE, st, launch_route(p, st));
-      if (logits_out)
-        CK(cudaMemcpyAsync(logits_out + (size_t)t0 * LS * c.n_experts, ctx->z_buf, (size_t)nt * LS * c.n_experts * 4,
-                           cudaMemcpyDeviceToDevice, st));
     }
   } else {
-    p.n_steps = n_steps, p.hidden = hidden, p.logits_in = logits_in;
+    p.n_steps = n_steps, p.hidden = hidden, p.logits_in = logits_in, p.n_partials = 1, p.partial_stride = 0;
     p.sel_idx = sel_idx, p.sel_w = sel_w, p.logits_out = logits_out;
     p.tok0 = (uint32_t)ctx->tok, p.cnt0 = (uint32_t)ctx->delta_cnt;
     TIMED(MCCE_K_ROUTE, st, launch_route(p, st));

@@ -20,7 +20,10 @@ struct RouteParams {
   int delta_mode, renorm;
   int hidden_bf16;
   const void* hidden;        // [n_steps,L,S,d] or null
-  const float* logits_in;    // [n_steps,L,S,E] or null
+  const float* logits_in;    // [n_steps,L,S,E] or null; n_partials such arrays, partial_stride elements apart,
+                             // are summed (the tensor-core router GEMM may split its reduction)
+  int n_partials;
+  size_t partial_stride;
   const float* Wr;           // [L,E,d]
   const float* fixed_delta;  // [L]
   uint32_t* stamp;           // [L,S,E]   0 = not resident, else recency key
@@ -71,7 +74,7 @@ bool router_gemm_applicable(const mcce_config& c);
 int router_gemm_steps_max();
 int router_gemm_plan(const mcce_config& c, const float* Wr, void* terms, RouterGemmPlan* plan, cudaStream_t st);
 cudaError_t router_gemm_launch(RouterGemmPlan& plan, const mcce_config& c, const void* hidden, int n_steps, float* Z,
-                               uint32_t* err, cudaStream_t st);
+                               int* k_split, uint32_t* err, cudaStream_t st);
 
 cudaError_t launch_route(const RouteParams& p, cudaStream_t st);
 cudaError_t launch_group(const GroupParams& p, cudaStream_t st);

@@ -146,7 +146,12 @@ __global__ void __launch_bounds__(kWarps * 32) route_kernel(const RouteParams p,
 #pragma unroll
       for (int i = 0; i < NE; ++i) {
         const int e = lane + 32 * i;
-        zr[i] = (active && e < E) ? __ldg(p.logits_in + row * E + e) : 0.f;
+        float z = 0.f;
+        if (active && e < E) {
+          z = __ldg(p.logits_in + row * E + e);
+          for (int q = 1; q < p.n_partials; ++q) z = __fadd_rn(z, __ldg(p.logits_in + q * p.partial_stride + row * E + e));
+        }
+        zr[i] = z;
       }
     }
     if (!active) continue;

@@ -12,6 +12,10 @@
 // every kPhaseSlabs K-slabs: the epilogue warps add each phase's two partial sums into fp32 registers
 // with round-to-nearest adds while the MMA warp continues in the other TMEM buffer.
 //
+// Speed: an MMA that accumulates into the accumulator of the previous MMA waits for it (~100 cycles at
+// these small N), so consecutive k-steps alternate between kAccSets independent accumulator sets and
+// the 12 MMAs of a K-slab form chains of at most four.
+//
 // Layout of the work: swapped GEMM as in the expert kernels -- router rows (experts) are MMA M (tiles of
 // 128, rows past E zero-filled by TMA at no memory cost), a block of streams is MMA N, the hidden
 // dimension is K in 64-column slabs.  Persistent CTAs walk (token, layer, expert tile, stream block)
@@ -26,18 +30,27 @@ using namespace tc;
 
 namespace {
 
-constexpr int kTileM = 128, kTileK = 64, kNSMax = 64, kXBox = 16, kThreads = 192, kStages = 4;
-constexpr uint32_t kABytes = kTileM * kTileK * 2;          // one bf16 term of the router tile: 16 KB
-constexpr uint32_t kBBytes = kNSMax * kTileK * 2;          // stream rows: 8 KB
-constexpr uint32_t kStageBytes = 3 * kABytes + kBBytes;    // 56 KB
-constexpr int kAccCols = 2 * kNSMax, kTmemCols = 2 * kAccCols; // per buffer: hi + mid/lo partial sums; 2 buffers
+constexpr int kTileM = 128, kTileK = 64, kNSMax = 64, kXBox = 16, kThreads = 192, kMaxStages = 12;
+constexpr uint32_t kRowBytes = kTileK * 2;                 // one 128-byte swizzle row
+// The stage ring.  A stage holds the three bf16 terms of a router slab -- only the RA rows that exist
+// (E rounded up to 8, at most 128) -- and the stream rows.  The MMA always reads 128 rows from a term's
+// start; rows past RA are whatever follows in the ring (finite or not, they only reach accumulator
+// rows of experts that do not exist), so the last 16 KB of the ring are never used as a stage start.
+constexpr uint32_t kRingBytes = 208 * 1024, kTermReadBytes = kTileM * kRowBytes;
+constexpr int kAccSets = 2;                                // independent accumulator sets (alternate k-steps)
+constexpr int kAccCols = 2 * kAccSets * kNSMax, kTmemCols = 2 * kAccCols;  // per buffer: sets x {hi, mid/lo}; 2 buffers
 constexpr int kPhaseSlabs = 4;                             // K-slabs (of 64) per accumulation phase
-constexpr size_t kSmemBytes = (size_t)kStages * kStageBytes + 1024 + 256;
+constexpr size_t kSmemBytes = (size_t)kRingBytes + 1024 + 256;
 
 struct GemmArgs {
   int L, S, E, d, n_steps, NS;
+  int RA;          // router rows per term tile actually loaded
+  int KS, kt_per;  // K-split: partial sums over kt_per slabs each
+  int n_stages;
+  uint32_t stage_bytes;
   int n_items;
-  float* Z;        // [n_steps, L, S, E]
+  float* Z;        // [KS][n_steps, L, S, E] partial logits
+  size_t z_stride; // elements between partials
   uint32_t* err;
 };
 struct GemmMaps {
@@ -46,16 +59,18 @@ struct GemmMaps {
 };
 
 struct GItem {
-  int l, mt, s0, row0;  // layer, expert tile, first stream, first hidden row (t*L + l)*S + s0
+  int l, mt, ks, s0, row0;  // layer, expert tile, K part, first stream, first hidden row (t*L + l)*S + s0
 };
 
 __device__ __forceinline__ GItem decode(const GemmArgs& a, int w) {
   const int SB = (a.S + a.NS - 1) / a.NS, MT = (a.E + kTileM - 1) / kTileM;
   GItem it;
   const int sb = w % SB;
-  it.mt = (w / SB) % MT;
-  it.l = (w / (SB * MT)) % a.L;
-  const int t = w / (SB * MT * a.L);
+  it.ks = (w / SB) % a.KS;
+  w /= SB * a.KS;
+  it.mt = w % MT;
+  it.l = (w / MT) % a.L;
+  const int t = w / (MT * a.L);
   it.s0 = sb * a.NS;
   it.row0 = (t * a.L + it.l) * a.S + it.s0;
   return it;
@@ -73,18 +88,20 @@ router_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs a) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_al = smem_raw + (smem_base - smem_u32(smem_raw));
-  uint64_t* bars = (uint64_t*)(smem_al + (size_t)kStages * kStageBytes);
-  const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * kStages;
-  const uint32_t bar_tfull = bar_empty + 8 * kStages, bar_tempty = bar_tfull + 16;
-  uint32_t* tmem_slot = (uint32_t*)(bars + 2 * kStages + 4);
+  uint64_t* bars = (uint64_t*)(smem_al + (size_t)kRingBytes);
+  const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * kMaxStages;
+  const uint32_t bar_tfull = bar_empty + 8 * kMaxStages, bar_tempty = bar_tfull + 16;
+  uint32_t* tmem_slot = (uint32_t*)(bars + 2 * kMaxStages + 4);
+  const uint32_t kStages = (uint32_t)a.n_stages, kStageBytes = a.stage_bytes;
+  const uint32_t kABytes = (uint32_t)a.RA * kRowBytes;
   volatile uint32_t* abort_flag = tmem_slot + 1;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int KT = a.d / kTileK;
+  const int KT = a.kt_per;
   const uint32_t n = (uint32_t)a.NS;   // MMA N: multiple of 16
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) {
+    for (int s = 0; s < kMaxStages; ++s) {
       mbar_init(bar_full + 8 * s, 1);
       mbar_init(bar_empty + 8 * s, 1);
     }
@@ -108,7 +125,7 @@ router_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs a) {
       const uint32_t tx = 3 * kABytes + n * kTileK * 2;
       for (int w = blockIdx.x; w < a.n_items && alive; w += gridDim.x) {
         const GItem it = decode(a, w);
-        for (int kt = 0; kt < KT; ++kt) {
+        for (int kt = it.ks * KT; kt < (it.ks + 1) * KT; ++kt) {
           if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, a.err, 11u)) {
             alive = false;
             break;
@@ -138,7 +155,7 @@ router_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs a) {
             break;
           }
           tc_fence_after();
-          const uint32_t d_hi = tmem_base + buf * kAccCols, d_lo = d_hi + kNSMax;
+          const uint32_t d_buf = tmem_base + buf * kAccCols;
           const int k1 = min(KT, k0 + kPhaseSlabs);
           for (int kt = k0; kt < k1; ++kt) {
             if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag, a.err, 13u)) {
@@ -150,7 +167,8 @@ router_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs a) {
 #pragma unroll
             for (int k = 0; k < kTileK / 16; ++k) {
               const uint64_t bd = smem_desc(sb + k * 32);
-              const uint32_t first = (kt == k0 && k == 0) ? 0u : 1u;
+              const uint32_t first = (kt == k0 && k < kAccSets) ? 0u : 1u;
+              const uint32_t d_hi = d_buf + (k % kAccSets) * 2 * kNSMax, d_lo = d_hi + kNSMax;
               umma_bf16(d_hi, smem_desc(sa + k * 32), bd, idesc, first);
               umma_bf16(d_lo, smem_desc(sa + kABytes + k * 32), bd, idesc, first);
               umma_bf16(d_lo, smem_desc(sa + 2 * kABytes + k * 32), bd, idesc, 1u);
@@ -184,12 +202,15 @@ router_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs a) {
 #pragma unroll
         for (int n0 = 0; n0 < kNSMax; n0 += 16) {
           if (n0 < a.NS) {
-            float hi[16], lo[16];
+            float hi[16], lo[16], hi1[16], lo1[16];
             tmem_ld16(t0 + n0, hi);
             tmem_ld16(t0 + kNSMax + n0, lo);
+            tmem_ld16(t0 + 2 * kNSMax + n0, hi1);
+            tmem_ld16(t0 + 3 * kNSMax + n0, lo1);
             tmem_ld_wait();
 #pragma unroll
-            for (int j = 0; j < 16; ++j) zacc[n0 + j] = __fadd_rn(zacc[n0 + j], __fadd_rn(hi[j], lo[j]));
+            for (int j = 0; j < 16; ++j)
+              zacc[n0 + j] = __fadd_rn(zacc[n0 + j], __fadd_rn(__fadd_rn(hi[j], hi1[j]), __fadd_rn(lo[j], lo1[j])));
           }
         }
         tc_fence_before();
@@ -199,7 +220,7 @@ router_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs a) {
       if (alive && e < a.E) {
 #pragma unroll
         for (int j = 0; j < kNSMax; ++j)
-          if (j < a.NS && it.s0 + j < a.S) a.Z[(size_t)(it.row0 + j) * a.E + e] = zacc[j];
+          if (j < a.NS && it.s0 + j < a.S) a.Z[it.ks * a.z_stride + (size_t)(it.row0 + j) * a.E + e] = zacc[j];
       }
     }
   }
@@ -231,6 +252,9 @@ __global__ void split_router_kernel(const float* W, __nv_bfloat16* out, size_t n
 
 }  // namespace
 
+// Router rows loaded per term tile: all 128 of a full tile, else E rounded up to the 8-row swizzle group.
+static int term_rows(int E) { return E >= kTileM ? kTileM : (E + 7) & ~7; }
+
 bool router_gemm_applicable(const mcce_config& c) { return c.hidden_dtype == MCCE_BF16 && c.d_model % kTileK == 0; }
 
 int router_gemm_steps_max() { return 8; }
@@ -245,7 +269,7 @@ int router_gemm_plan(const mcce_config& c, const float* Wr, void* terms, RouterG
   if (!fn) return MCCE_ECUDA;
   const cuuint64_t dims[3] = {(cuuint64_t)c.d_model, (cuuint64_t)c.n_experts, (cuuint64_t)3 * c.n_layers};
   const cuuint64_t strides[2] = {(cuuint64_t)c.d_model * 2, (cuuint64_t)c.d_model * 2 * c.n_experts};
-  const cuuint32_t box[3] = {(cuuint32_t)kTileK, (cuuint32_t)kTileM, 1};
+  const cuuint32_t box[3] = {(cuuint32_t)kTileK, (cuuint32_t)term_rows(c.n_experts), 1};
   const cuuint32_t estr[3] = {1, 1, 1};
   if (fn(&plan->w, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, terms, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
          CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -258,7 +282,7 @@ int router_gemm_plan(const mcce_config& c, const float* Wr, void* terms, RouterG
 }
 
 cudaError_t router_gemm_launch(RouterGemmPlan& plan, const mcce_config& c, const void* hidden, int n_steps, float* Z,
-                               uint32_t* err, cudaStream_t st) {
+                               int* k_split, uint32_t* err, cudaStream_t st) {
   static int sms = 0;
   if (!sms) {
     int dev = 0;
@@ -293,8 +317,25 @@ cudaError_t router_gemm_launch(RouterGemmPlan& plan, const mcce_config& c, const
   while (ns > 16 && n_steps * c.n_layers * mt * ((c.n_streams + ns - 1) / ns) < sms / 2) ns /= 2;
   ns = (ns + 15) & ~15;
   a.NS = ns;
-  a.n_items = n_steps * c.n_layers * mt * ((c.n_streams + ns - 1) / ns);
-  a.Z = Z, a.err = err;
+  // split the reduction over up to four CTAs per tile while SMs would otherwise idle; the partial
+  // logits are summed by the routing tail.  The logits buffer has router_gemm_steps_max() slots.
+  const int kt = c.d_model / kTileK;
+  const int items = n_steps * c.n_layers * mt * ((c.n_streams + ns - 1) / ns);
+  int ks = 1;
+  double best = (double)((items + sms - 1) / sms);   // rounds of the persistent grid, in whole-tile units
+  for (int cand = 2; cand <= 4; cand *= 2) {
+    if (kt % cand || kt / cand < 4 || n_steps * cand > router_gemm_steps_max()) break;
+    const double cost = (double)((items * cand + sms - 1) / sms) / cand;
+    if (cost < best - 1e-9) best = cost, ks = cand;
+  }
+  a.KS = ks, a.kt_per = kt / ks;
+  a.n_items = items * ks;
+  a.RA = term_rows(c.n_experts);
+  a.stage_bytes = (uint32_t)(3 * a.RA + ns) * kRowBytes;
+  a.n_stages = (int)((kRingBytes - kTermReadBytes) / a.stage_bytes);
+  if (a.n_stages > kMaxStages) a.n_stages = kMaxStages;
+  a.Z = Z, a.z_stride = (size_t)rows * c.n_experts, a.err = err;
+  *k_split = ks;
   GemmMaps m;
   m.w = plan.w, m.x = plan.x;
   const int grid = a.n_items < sms ? a.n_items : sms;
