@@ -271,7 +271,10 @@ def main_arm(args):
     rows = wl.L * wl.S * (wl.K + wl.n_shared)
     esz = 2 if wl.bf16 else 4
     bytes_up = touched * 2 * wl.d * wl.I * esz + rows * wl.d * esz + rows * wl.I * esz
-    bytes_down = touched * wl.d * wl.I * esz + rows * wl.I * esz + rows * wl.d * 4
+    # down projection: weights + H rows; the tensor path adds into y (L*S*d fp32) in its epilogue, the
+    # fp32-pipe path writes one fp32 row per (pair) for a separate combine pass
+    bytes_down = touched * wl.d * wl.I * esz + rows * wl.I * esz + (
+        wl.L * wl.S * wl.d * 4 if _uses_tensor(eng) else rows * wl.d * 4)
     up_ms, up_n = prof["ffn_up"]
     peak, peak_src = measured_hbm_peak()
     achieved = bytes_up / (up_ms / max(1, up_n) * 1e-3) / 1e9

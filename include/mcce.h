@@ -117,7 +117,9 @@ int mcce_route_step(mcce_ctx* ctx, int32_t n_steps, const void* hidden, const fl
  * SwiGLU experts group by group and combines y = sum_k w_k E_sel_k(x) (slot order) + shared experts.
  *   hidden DEVICE hidden_dtype [L,S,d]; sel_idx DEVICE int32 [L,S,K]; sel_w DEVICE fp32 [L,S,K];
  *   y DEVICE fp32 [L,S,d] out.
- * With bf16 weights the intermediate silu(g)*u is rounded to bf16 before the down projection. */
+ * With bf16 weights the intermediate silu(g)*u is rounded to bf16 before the down projection.  On the
+ * tensor-core path the K + n_shared terms of a stream are added into y with fp32 atomic adds in no fixed
+ * order, so the last bits of y may differ between runs (the fp32-pipe path sums in slot order). */
 int mcce_moe_forward(mcce_ctx* ctx, const void* hidden, const int32_t* sel_idx, const float* sel_w,
                      float* y, void* cuda_stream);
 

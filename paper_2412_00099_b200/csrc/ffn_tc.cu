@@ -12,7 +12,9 @@
 // One CTA per SM walks a static list of (layer, expert, 128-row tile) items.  Warp 0 issues TMA loads
 // (128B-swizzled 64-column slabs of the weight tile and of the token rows) into a ring of shared-memory
 // stages, warp 1 issues tcgen05.mma into one of two TMEM accumulator buffers, warps 2-5 drain the other
-// buffer with tcgen05.ld, apply the epilogue and write the result.  Every wait on an mbarrier is bounded:
+// buffer with tcgen05.ld and apply the epilogue: SwiGLU and a bf16 store of H (up), or the weighted
+// combine of Eq. 1 straight into y with fp32 atomic adds (down; y is zeroed first, and since the order
+// of a stream's K + shared addends is not fixed, the last bits of y may differ from run to run).  Every wait on an mbarrier is bounded:
 // on a timeout the CTA records an error word, stops, releases its TMEM and returns.
 #include <cuda.h>
 
@@ -46,8 +48,10 @@ struct TcArgs {
   int L, S, E, K, n_sh, d, I;
   int n_items;
   const int32_t* offsets;
+  const int32_t* perm;   // [L, S*K] position -> pair, for the fused combine of the down kernel
+  const float* sel_w;    // [L, S, K]
   __nv_bfloat16* H;
-  float* O;
+  float* y;              // [L, S, d], zeroed before the down kernel; receives w * E_i(x) by fp32 atomic adds
   uint32_t* err;
 };
 
@@ -67,6 +71,7 @@ struct Item {
   int xrow;       // first token row in the activation tensor map
   size_t orow;    // first row in H / O
   int col0;       // first output column (= weight row inside the expert) of this tile
+  int l;          // layer
   bool shared;
 };
 
@@ -81,6 +86,7 @@ __device__ __forceinline__ Item decode(const TcArgs& a, int w) {
   const int per_layer = items_per_layer(a.E, a.n_sh, a.S, RT);
   const int l = w / per_layer, wl = w % per_layer;
   Item it;
+  it.l = l;
   if (wl < a.E * RT) {
     const int g = wl / RT;
     it.col0 = (wl % RT) * kTileM;
@@ -243,10 +249,28 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, const TcArgs a) {
               }
             }
           } else {
+            // Eq. 1 combine, fused: y[l, s, :] += w * o.  Lane j looks up the stream and weight of token
+            // n0 + j; all lanes then add their column of that token (32 consecutive floats per warp).
+            int my_dst = -1;
+            float my_w = 0.f;
+            if (lane < 16 && n0 + lane < ntok) {
+              const size_t r = it.orow + c0 + n0 + lane;
+              if (it.shared) {
+                my_dst = it.l * a.S + (int)((r - (size_t)a.L * a.S * a.K) % a.S);
+                my_w = 1.f;
+              } else {
+                const int pair = __ldg(a.perm + r);
+                my_dst = it.l * a.S + pair / a.K;
+                my_w = __ldg(a.sel_w + (size_t)it.l * a.S * a.K + pair);
+              }
+            }
             tmem_ld_wait();
 #pragma unroll
-            for (int j = 0; j < 16; ++j)
-              if (n0 + j < ntok) a.O[(it.orow + c0 + n0 + j) * a.d + col] = g[j];
+            for (int j = 0; j < 16; ++j) {
+              const int dst = __shfl_sync(0xffffffffu, my_dst, j);
+              const float w = __shfl_sync(0xffffffffu, my_w, j);
+              if (dst >= 0) atomicAdd(a.y + (size_t)dst * a.d + col, w * g[j]);
+            }
           }
         }
         tc_fence_before();
@@ -300,7 +324,7 @@ cudaError_t launch(const TcMaps& maps, const FfnParams& p, uint32_t* err, cudaSt
   TcArgs a;
   a.L = p.L, a.S = p.S, a.E = p.E, a.K = p.K, a.n_sh = p.n_sh, a.d = p.d, a.I = p.I;
   a.n_items = p.L * items_per_layer(p.E, p.n_sh, p.S, (UP ? p.I : p.d) / kTileM);
-  a.offsets = p.offsets, a.H = (__nv_bfloat16*)p.H, a.O = p.O, a.err = err;
+  a.offsets = p.offsets, a.perm = p.perm, a.sel_w = p.sel_w, a.H = (__nv_bfloat16*)p.H, a.y = p.y, a.err = err;
   const int grid = a.n_items < sms ? a.n_items : sms;
   ffn_tc_kernel<UP><<<grid, kThreads, Cfg<UP>::kSmemBytes, st>>>(maps, a);
   return cudaGetLastError();

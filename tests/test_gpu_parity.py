@@ -270,7 +270,9 @@ def test_decode_step_from_host_buffers():
         xd = xh.cuda()
         sel, w = ref.route_step(hidden=xd[None])
         y = ref.moe_forward(xd, sel[0], w[0])
-        assert torch.equal(sh, sel[0].cpu()) and torch.equal(yh, y.cpu())
+        assert torch.equal(sh, sel[0].cpu())
+        # y is summed with fp32 atomics on the tensor path: same terms, order not fixed
+        assert torch.allclose(yh, y.cpu(), rtol=1e-5, atol=1e-6)
 
 
 # ---- argument checking: errors come back as codes, nothing is launched ------------------------------------
