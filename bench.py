@@ -287,6 +287,16 @@ def main_arm(args):
     kernels = {k: {"ms_per_step": v[0] / K, "launches": v[1]} for k, v in prof.items()}
     dn_ms, dn_n = prof["ffn_down"]
     kernels["ffn_down"]["achieved_gbs"] = bytes_down / (dn_ms / max(1, dn_n) * 1e-3) / 1e9
+    # routing (logits + fused tail): hidden rows, the router once per layer, cache state in and out, results
+    EW = (wl.E + 31) // 32
+    bytes_route = wl.L * wl.S * (wl.d * esz + 2 * (wl.E * 4 + EW * 4 + 12) + wl.K * 8) + wl.L * wl.E * wl.d * 4
+    route_ms = (prof["route"][0] + prof["route_gemm"][0]) / K
+    kernels["route"]["achieved_gbs_with_gemm"] = bytes_route / (route_ms * 1e-3) / 1e9
+    kernels["route"]["algorithmic_bytes"] = bytes_route
+    # grouping + gather: selections in, offsets / permutation out, hidden rows copied into expert order
+    bytes_group = wl.L * wl.S * wl.K * (4 + 8) + 2 * wl.L * wl.S * wl.K * wl.d * esz
+    kernels["gather"]["achieved_gbs_with_group"] = bytes_group / (
+        (prof["group"][0] + prof["gather"][0]) / K * 1e-3) / 1e9
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
             "ms_per_step": ms_total / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,

@@ -37,7 +37,7 @@ constexpr uint32_t kBBytes = kNMax * kTileK * 2;    // 16 KB
 
 template <bool UP>
 struct Cfg {
-  static constexpr int kStages = UP ? 4 : 6;
+  static constexpr int kStages = UP ? 4 : 7;
   static constexpr uint32_t kStageBytes = (UP ? 2 : 1) * kABytes + kBBytes;
   static constexpr int kAccCols = UP ? 2 * kNMax : kNMax;   // TMEM columns per accumulator buffer
   static constexpr int kTmemCols = 2 * kAccCols;            // two buffers: 512 / 256
@@ -150,8 +150,10 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, const TcArgs a) {
     if (lane == 0) {
       uint32_t stage = 0, phase = 0;
       bool alive = true;
+      Item nxt = decode<UP>(a, min((int)blockIdx.x, a.n_items - 1));
       for (int w = blockIdx.x; w < a.n_items && alive; w += gridDim.x) {
-        const Item it = decode<UP>(a, w);
+        const Item it = nxt;   // the next item's group offsets are fetched while this one streams
+        if (w + (int)gridDim.x < a.n_items) nxt = decode<UP>(a, w + gridDim.x);
         const CUtensorMap* mw0 = it.shared ? &maps.sw0 : &maps.w0;
         const CUtensorMap* mw1 = it.shared ? &maps.sw1 : &maps.w1;
         const CUtensorMap* mx = it.shared ? &maps.xs : &maps.x;
@@ -181,8 +183,10 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, const TcArgs a) {
     if (lane == 0) {
       uint32_t stage = 0, phase = 0, acc_iter = 0;
       bool alive = true;
+      Item nxt = decode<UP>(a, min((int)blockIdx.x, a.n_items - 1));
       for (int w = blockIdx.x; w < a.n_items && alive; w += gridDim.x) {
-        const Item it = decode<UP>(a, w);
+        const Item it = nxt;
+        if (w + (int)gridDim.x < a.n_items) nxt = decode<UP>(a, w + gridDim.x);
         for (int c0 = 0; c0 < it.m && alive; c0 += kNMax, ++acc_iter) {
           const uint32_t n = (uint32_t)(min(kNMax, it.m - c0) + 15) & ~15u;
           const uint32_t idesc = instr_desc(n);
@@ -221,8 +225,10 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, const TcArgs a) {
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
     uint32_t acc_iter = 0;
     bool alive = true;
+    Item nxt = decode<UP>(a, min((int)blockIdx.x, a.n_items - 1));
     for (int w = blockIdx.x; w < a.n_items && alive; w += gridDim.x) {
-      const Item it = decode<UP>(a, w);
+      const Item it = nxt;
+      if (w + (int)gridDim.x < a.n_items) nxt = decode<UP>(a, w + gridDim.x);
       const int col = it.col0 + quad * 32 + lane;      // output feature handled by this thread
       for (int c0 = 0; c0 < it.m && alive; c0 += kNMax, ++acc_iter) {
         const int ntok = min(kNMax, it.m - c0);
