@@ -41,7 +41,13 @@ typedef struct {
   int32_t delta_mode;                                  /* 0 running mean (Eq. 8), 1 fixed per layer */
   int32_t renorm;                                      /* 1: weights renormalised over the selected */
   int32_t dtype;                                       /* 0: fp32 everywhere, 1: bf16 hidden+weights */
+  int32_t rerank_mode;                                 /* 0 Cache-Prior (Eq. 7), 1 Max-Rank (Alg. 1),
+                                                          2 Cumsum-Threshold (Alg. 2)               */
+  int32_t max_rank;                                    /* M of Algorithm 1                          */
+  float cum_threshold;                                 /* p of Algorithm 2                          */
 } orc_config;
+
+void orc_max_rank(const int32_t* r, int n, const uint8_t* in_cache, int M, int J, int32_t* out);
 
 /* ---------------------------------------------------------------------------------------------- */
 /* small helpers                                                                                   */
@@ -168,7 +174,34 @@ void orc_route_slab(const orc_config* c, const float* z_all /*[L,S,E]*/,
       /* r' = argsort(z'); the first K are selected. */
       int32_t rank[ORC_MAX_E];
       const int need = K < E ? K + 1 : K;
-      top_by_value(zp, E, need, rank);
+      float cum_margin = INFINITY;
+      if (c->rerank_mode == 0) {
+        top_by_value(zp, E, need, rank);
+      } else {
+        /* The two baselines rerank the router's own ranking r with the list operator of Sec. 3.1. */
+        int32_t r[ORC_MAX_E];
+        uint8_t in_cache[ORC_MAX_E];
+        top_by_value(z, E, E, r);
+        for (int e = 0; e < E; ++e) in_cache[e] = stamp[e] != 0;
+        int M = c->max_rank;
+        if (c->rerank_mode == 2) {
+          /* Algorithm 2: M = smallest count of top-ranked experts whose probabilities reach p. */
+          double denom = 0.0;
+          for (int e = 0; e < E; ++e) denom += exp((double)z[e] - (double)zmax);
+          float p_cum = 0.0f;
+          M = 0;
+          while (p_cum < c->cum_threshold && M < E) {
+            M += 1;
+            const float wr = (float)(exp((double)z[r[M - 1]] - (double)zmax) / denom);
+            const float before = p_cum;
+            p_cum = p_cum + wr;
+            /* distance of the threshold from the two partial sums that decided M */
+            if (p_cum >= c->cum_threshold)
+              cum_margin = fminf(p_cum - c->cum_threshold, c->cum_threshold - before);
+          }
+        }
+        orc_max_rank(r, E, in_cache, M, J, rank);
+      }
       for (int k = 0; k < K; ++k) sel[k] = rank[k];
 
       /* Expert weights: softmax of the UNMODIFIED logits (Eq. 3), optionally renormalised over
@@ -234,7 +267,15 @@ void orc_route_slab(const orc_config* c, const float* z_all /*[L,S,E]*/,
         /* the smallest gap that decided something: K-th vs (K+1)-th of z', J-th vs (J+1)-th of z,
            and neighbours in the in-token touch order */
         float m = INFINITY;
-        if (K < E) m = fminf(m, zp[rank[K - 1]] - zp[rank[K]]);
+        if (K < E && c->rerank_mode == 0) m = fminf(m, zp[rank[K - 1]] - zp[rank[K]]);
+        if (c->rerank_mode != 0) {
+          /* any two neighbours of the router's ranking may swap; the cumulative threshold may fall
+             on either side */
+          int32_t r[ORC_MAX_E];
+          top_by_value(z, E, E, r);
+          for (int i = 0; i + 1 < E; ++i) m = fminf(m, z[r[i]] - z[r[i + 1]]);
+          m = fminf(m, cum_margin);
+        }
         if (J > 0 && J < E) {
           int32_t tj[ORC_MAX_E];
           top_by_value(z, E, J + 1, tj);

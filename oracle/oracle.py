@@ -33,7 +33,8 @@ class _Cfg(C.Structure):
     _fields_ = [(n, C.c_int32) for n in
                 ("n_layers", "n_experts", "top_k", "top_j", "n_shared", "d_model", "d_ff",
                  "cache_capacity", "n_streams")] + [
-        ("lam", C.c_float), ("delta_mode", C.c_int32), ("renorm", C.c_int32), ("dtype", C.c_int32)]
+        ("lam", C.c_float), ("delta_mode", C.c_int32), ("renorm", C.c_int32), ("dtype", C.c_int32),
+        ("rerank_mode", C.c_int32), ("max_rank", C.c_int32), ("cum_threshold", C.c_float)]
 
 
 _lib = None
@@ -68,11 +69,15 @@ class OracleConfig:
     delta_mode: int = 0
     renorm: int = 1
     dtype: int = 1  # 0 fp32, 1 bf16 (uint16 storage)
+    rerank_mode: int = 0  # 0 Cache-Prior, 1 Max-Rank, 2 Cumsum-Threshold
+    max_rank: int = 0
+    cum_threshold: float = 0.0
 
     def c(self) -> _Cfg:
         return _Cfg(self.n_layers, self.n_experts, self.top_k, self.top_j, self.n_shared,
                     self.d_model, self.d_ff, self.cache_capacity, self.n_streams, self.lam,
-                    self.delta_mode, self.renorm, self.dtype)
+                    self.delta_mode, self.renorm, self.dtype, self.rerank_mode, self.max_rank,
+                    self.cum_threshold)
 
 
 def _split(n: int, parts: int):

@@ -485,3 +485,75 @@ def test_initial_cache_state_is_older_than_any_touch():
     o.route(np.array([[[0, 0, 9, 0, 0, 0]]], np.float32))       # hit on 2
     assert o.order()[0, 0].tolist() == [2, 0, 4]
     assert o.stats()[0].tolist() == [2, 2, 1, 1]
+
+
+# ---- the two baseline rerankers as routing modes (Algorithms 1 and 2) -------------------------------
+def make_mode(mode, E, K, J, C, M=0, p=0.0, lam=0.5, L=1, S=3):
+    cfg = orc.OracleConfig(L, E, K, J, 0, 16, 8, C, S, lam, 0, 1, 0, mode, M, p)
+    return orc.Oracle(cfg)
+
+
+def py_max_rank_select(z, resident, M, J, K):
+    r = plain_topk(z, len(z)).tolist()
+    step1 = py_promote([e for e in r[:M] if resident[e]], r)
+    return py_promote(r[:J], step1)[:K]
+
+
+@pytest.mark.parametrize("M", [0, 2, 4, 9])
+@pytest.mark.parametrize("J", [0, 1, 2])
+def test_max_rank_mode_follows_algorithm_1(M, J):
+    rng = np.random.default_rng(100 + 10 * M + J)
+    E, K, C = 9, 3, 4
+    o = make_mode(1, E, K, J, C, M=M)
+    for z in ar1_logits(rng, 60, 1, 3, E):
+        resident = (o.stamp != 0).copy()
+        sel, _ = o.route(z)
+        for s in range(3):
+            assert sel[0, s].tolist() == py_max_rank_select(z[0, s], resident[0, s], M, J, K)
+            if M == 0:
+                assert sel[0, s].tolist() == plain_topk(z[0, s], K).tolist()     # nothing may be promoted
+
+
+@pytest.mark.parametrize("J", [0, 1, 2])
+def test_max_rank_over_all_ranks_is_the_saturated_cache_prior(J):
+    """Two independent routes through the oracle: Eq. 7 with a bias beyond the logit range, and the list
+    operator with M = N.  Same trace, same cache evolution, same selections."""
+    rng = np.random.default_rng(7 + J)
+    E, K, C = 10, 3, 5
+    a = make_mode(0, E, K, J, C, lam=50.0)
+    b = make_mode(1, E, K, J, C, M=E)
+    for z in ar1_logits(rng, 80, 1, 3, E):
+        sa, wa = a.route(z)
+        sb, wb = b.route(z)
+        assert np.array_equal(sa, sb) and np.array_equal(wa, wb)
+    assert np.array_equal(a.stamp, b.stamp) and np.array_equal(a.counters, b.counters)
+
+
+@pytest.mark.parametrize("p", [0.0, 0.3, 0.6, 0.9, 1.5])
+def test_cumsum_mode_follows_algorithm_2(p):
+    rng = np.random.default_rng(int(p * 10) + 200)
+    E, K, J, C = 8, 2, 1, 4
+    o = make_mode(2, E, K, J, C, p=p)
+    for z in ar1_logits(rng, 60, 1, 3, E):
+        resident = (o.stamp != 0).copy()
+        sel, _, margin, _ = o.route(z, want_margin=True)
+        for s in range(3):
+            zz = z[0, s]
+            w = torch.softmax(torch.tensor(zz, dtype=torch.float64), 0).numpy()
+            r = plain_topk(zz, E).tolist()
+            cum = np.cumsum(w[r])
+            M = int(np.searchsorted(cum, p, side="left")) + 1 if p > 0 else 0
+            M = min(M, E)
+            if margin[0, s] < 1e-6:
+                continue                      # threshold within rounding of a partial sum: either M is right
+            assert sel[0, s].tolist() == py_max_rank_select(zz, resident[0, s], M, J, K)
+    if p == 0.0:
+        assert o.stats()[0][2] == make_and_run_plain(E, K, J, C, int(p * 10) + 200)
+
+
+def make_and_run_plain(E, K, J, C, seed):
+    rng = np.random.default_rng(seed)
+    o = make_mode(0, E, K, J, C, lam=0.0)
+    for z in ar1_logits(rng, 60, 1, 3, E):
+        o.route(z)
+    return o.stats()[0][2]
