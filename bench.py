@@ -46,6 +46,10 @@ def parse_args():
     ap.add_argument("--lam", type=float, default=None, help="promotion strength lambda")
     ap.add_argument("--layers", type=int, default=None,
                     help="fewer layers than the workload has (small cases for profiler captures; not a bench line)")
+    ap.add_argument("--rerank", default="prior", choices=["prior", "maxrank", "cumsum"],
+                    help="Cache-Prior (Eq. 7, the headline), or the Max-Rank / Cumsum-Threshold baselines")
+    ap.add_argument("--max-rank", type=int, default=None, help="M of Max-Rank (default 2K)")
+    ap.add_argument("--cum-p", type=float, default=0.5, help="p of Cumsum-Threshold")
     ap.add_argument("--impl", default="mcce", choices=["mcce", "reference"])
     ap.add_argument("--ffn", default="auto", choices=["auto", "simt", "tensor"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -198,7 +202,10 @@ def main_arm(args):
     # streams are independent: rank r owns its own S streams (weak scaling), distinguished by the seed
     seed = replica_seed(wl.seed, rank)
     ffn_impl = {"auto": mb.FFN_AUTO, "simt": mb.FFN_SIMT, "tensor": mb.FFN_TENSOR}[args.ffn]
-    eng = mb.engine_for(wl, ffn_impl=ffn_impl, device=local)
+    rerank = {"prior": mb.RERANK_CACHE_PRIOR, "maxrank": mb.RERANK_MAX_RANK, "cumsum": mb.RERANK_CUMSUM}[args.rerank]
+    max_rank = min(wl.E, args.max_rank if args.max_rank is not None else 2 * wl.K)
+    eng = mb.engine_for(wl, ffn_impl=ffn_impl, device=local, rerank_mode=rerank, max_rank=max_rank,
+                        cum_threshold=args.cum_p)
     wdt = torch.bfloat16 if wl.bf16 else torch.float32
 
     # ---- weights, generated on the device ------------------------------------------------------------
@@ -304,6 +311,9 @@ def main_arm(args):
             "config": config_of(wl, {"l2": "inputs larger than L2: %.1f GB of expert weights streamed per step"
                                            % ((bytes_up + bytes_down) / 1e9),
                                      "ffn_path": "tensor" if _uses_tensor(eng) else "simt",
+                                     "rerank": args.rerank if args.rerank == "prior" else (
+                                         "maxrank M=%d" % max_rank if args.rerank == "maxrank"
+                                         else "cumsum p=%g" % args.cum_p),
                                      "experts_touched_per_step": touched}),
             "miss_rate": misses / max(1, selections), "roofline": roofline, "kernels": kernels,
             "gpu_launches": int(sum(v[1] for v in prof.values())), "clocks": clocks}

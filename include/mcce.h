@@ -40,6 +40,12 @@ enum {
 enum { MCCE_F32 = 0, MCCE_BF16 = 1 };
 enum { MCCE_DELTA_RUNNING = 0, MCCE_DELTA_FIXED = 1 };
 enum { MCCE_FFN_AUTO = 0, MCCE_FFN_SIMT = 1, MCCE_FFN_TENSOR = 2 };
+/* How the router's ranking r is changed in favour of cached experts (Sec. 3):
+ * CACHE_PRIOR  Eq. 7, the paper's main method: rank by z' = z + lambda*Delta_avg*m~_t;
+ * MAX_RANK     Algorithm 1: promote(r[:J]; promote(r[:M] ∩ C; r)) with M = max_rank;
+ * CUMSUM       Algorithm 2: the same with M = the smallest number of top-ranked experts whose router
+ *              probabilities sum to at least cum_threshold. */
+enum { MCCE_RERANK_CACHE_PRIOR = 0, MCCE_RERANK_MAX_RANK = 1, MCCE_RERANK_CUMSUM = 2 };
 
 typedef struct mcce_ctx mcce_ctx; /* opaque; host memory owned by the library */
 
@@ -63,6 +69,9 @@ typedef struct {
   int32_t weight_dtype;   /* expert weights; must equal hidden_dtype                             */
   int32_t ffn_impl;       /* MCCE_FFN_AUTO picks the tensor-core path when it applies            */
   int32_t device;         /* CUDA device ordinal                                                 */
+  int32_t rerank_mode;    /* MCCE_RERANK_*; lambda / delta_mode only matter for CACHE_PRIOR      */
+  int32_t max_rank;       /* M of Algorithm 1, 0..E (MAX_RANK only)                              */
+  float cum_threshold;    /* p of Algorithm 2, >= 0 (CUMSUM only)                                */
 } mcce_config;
 
 typedef struct {

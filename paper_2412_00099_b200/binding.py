@@ -17,6 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libmcce.so")
 F32, BF16 = 0, 1
 DELTA_RUNNING, DELTA_FIXED = 0, 1
 FFN_AUTO, FFN_SIMT, FFN_TENSOR = 0, 1, 2
+RERANK_CACHE_PRIOR, RERANK_MAX_RANK, RERANK_CUMSUM = 0, 1, 2
 
 EXPORTS = [
     "mcce_workspace_bytes", "mcce_create", "mcce_destroy", "mcce_set_router", "mcce_set_experts", "mcce_reset",
@@ -31,7 +32,8 @@ class Config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("n_layers", "n_experts", "top_k", "top_j", "n_shared", "d_model", "d_ff",
                                          "cache_capacity", "n_streams")] + [
         ("lam", C.c_float), ("delta_mode", C.c_int32), ("renorm", C.c_int32), ("hidden_dtype", C.c_int32),
-        ("weight_dtype", C.c_int32), ("ffn_impl", C.c_int32), ("device", C.c_int32)]
+        ("weight_dtype", C.c_int32), ("ffn_impl", C.c_int32), ("device", C.c_int32),
+        ("rerank_mode", C.c_int32), ("max_rank", C.c_int32), ("cum_threshold", C.c_float)]
 
 
 class Stats(C.Structure):
@@ -114,12 +116,12 @@ class Engine:
     """One mcce context: the cache state of every (stream, layer) plus borrowed weights."""
 
     def __init__(self, *, L, E, K, J, n_shared, d, I, C_cap, S, lam, delta_mode=DELTA_RUNNING, renorm=1, dtype=BF16,
-                 ffn_impl=FFN_AUTO, device=0):
+                 ffn_impl=FFN_AUTO, device=0, rerank_mode=RERANK_CACHE_PRIOR, max_rank=0, cum_threshold=0.0):
         if not torch.cuda.is_available():
             raise McceError("no CUDA device: this library has no CPU path")
         self.lib = load()
         self.cfg = Config(L, E, K, J, n_shared, d, I, C_cap, S, lam, delta_mode, renorm, dtype, dtype, ffn_impl,
-                          device)
+                          device, rerank_mode, max_rank, cum_threshold)
         self.device = torch.device("cuda", device)
         nbytes = self.lib.mcce_workspace_bytes(C.byref(self.cfg))
         if nbytes == 0:

@@ -68,6 +68,9 @@ bool valid(const mcce_config* c) {
   if (c->ffn_impl < MCCE_FFN_AUTO || c->ffn_impl > MCCE_FFN_TENSOR) return false;
   if (c->ffn_impl == MCCE_FFN_TENSOR && !tc_applicable(*c)) return false;
   if (c->device < 0) return false;
+  if (c->rerank_mode < MCCE_RERANK_CACHE_PRIOR || c->rerank_mode > MCCE_RERANK_CUMSUM) return false;
+  if (c->rerank_mode == MCCE_RERANK_MAX_RANK && (c->max_rank < 0 || c->max_rank > c->n_experts)) return false;
+  if (c->rerank_mode == MCCE_RERANK_CUMSUM && !(c->cum_threshold >= 0.f)) return false;
   return true;
 }
 
@@ -304,6 +307,7 @@ extern "C" int mcce_route_step(mcce_ctx* ctx, int32_t n_steps, const void* hidde
   RouteParams p;
   p.L = c.n_layers, p.S = c.n_streams, p.E = c.n_experts, p.K = c.top_k, p.J = c.top_j, p.C = c.cache_capacity;
   p.d = c.d_model, p.lambda = c.lambda, p.delta_mode = c.delta_mode, p.renorm = c.renorm;
+  p.rerank_mode = c.rerank_mode, p.max_rank = c.max_rank, p.cum_threshold = c.cum_threshold;
   p.hidden_bf16 = c.hidden_dtype == MCCE_BF16;
   p.Wr = ctx->Wr, p.fixed_delta = ctx->fixed_delta;
   p.stamp = ctx->stamp, p.ever = ctx->ever, p.sum_range = ctx->sum_range, p.miss = ctx->miss, p.cold = ctx->cold;

@@ -18,6 +18,8 @@ struct RouteParams {
   int n_steps;
   float lambda;
   int delta_mode, renorm;
+  int rerank_mode, max_rank;  // MCCE_RERANK_*; M of Algorithm 1
+  float cum_threshold;        // p of Algorithm 2
   int hidden_bf16;
   const void* hidden;        // [n_steps,L,S,d] or null
   const float* logits_in;    // [n_steps,L,S,E] or null; n_partials such arrays, partial_stride elements apart,

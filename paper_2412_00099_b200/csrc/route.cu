@@ -195,12 +195,58 @@ __global__ void __launch_bounds__(kWarps * 32) route_kernel(const RouteParams p,
         mt |= 1u << (e >> 5);
       }
     }
-    uint32_t kp[NE];
+    uint32_t kp[NE];   // selection key of every expert: the K largest are selected, in this order
+    if (p.rerank_mode == MCCE_RERANK_CACHE_PRIOR) {
 #pragma unroll
-    for (int i = 0; i < NE; ++i) {
-      const bool valid = lane + 32 * i < E;
-      const float zp = ((mt >> i) & 1u) ? __fadd_rn(zr[i], bias) : zr[i];
-      kp[i] = valid ? okey(zp) : 0u;
+      for (int i = 0; i < NE; ++i) {
+        const bool valid = lane + 32 * i < E;
+        const float zp = ((mt >> i) & 1u) ? __fadd_rn(zr[i], bias) : zr[i];
+        kp[i] = valid ? okey(zp) : 0u;
+      }
+    } else {
+      // ---- Algorithms 1 and 2: promote(r[:J]; promote(r[:M] ∩ C; r)) on the router's own ranking r ------
+      // rank of every expert in r (value descending, index ascending), by comparison with all others
+      uint32_t rk[NE];
+#pragma unroll
+      for (int i = 0; i < NE; ++i) rk[i] = 0u;
+      for (int i2 = 0; i2 < NE; ++i2) {
+        for (int src = 0; src < 32; ++src) {
+          const int eo = src + 32 * i2;
+          if (eo >= E) break;
+          const uint32_t ko = __shfl_sync(kFull, key[i2], src);
+#pragma unroll
+          for (int i = 0; i < NE; ++i) rk[i] += (ko > key[i] || (ko == key[i] && eo < lane + 32 * i)) ? 1u : 0u;
+        }
+      }
+      int M = p.max_rank;
+      if (p.rerank_mode == MCCE_RERANK_CUMSUM) {
+        // Algorithm 2: walk down the ranking, summing router probabilities until they reach the threshold
+        float pr[NE], loc = 0.f;
+#pragma unroll
+        for (int i = 0; i < NE; ++i) {
+          pr[i] = lane + 32 * i < E ? expf(zr[i] - zmax) : 0.f;
+          loc += pr[i];
+        }
+        const float inv_all = warp_sum(loc);
+        float p_cum = 0.f;
+        M = 0;
+        while (p_cum < p.cum_threshold && M < E) {
+          float wv = 0.f;
+          bool own = false;   // exactly one lane holds the expert of rank M
+#pragma unroll
+          for (int i = 0; i < NE; ++i)
+            if (lane + 32 * i < E && rk[i] == (uint32_t)M) wv = pr[i] / inv_all, own = true;
+          wv = __shfl_sync(kFull, wv, __ffs(__ballot_sync(kFull, own)) - 1);
+          p_cum = __fadd_rn(p_cum, wv);
+          ++M;
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < NE; ++i) {
+        const bool valid = lane + 32 * i < E;
+        const uint32_t cls = rk[i] < (uint32_t)p.J ? 0u : ((rk[i] < (uint32_t)M && ((resb >> i) & 1u)) ? 1u : 2u);
+        kp[i] = valid ? 0x7fffffffu - ((cls << 16) | rk[i]) : 0u;
+      }
     }
 
     // ---- top-K of z' (rank order); lane r keeps the r-th selected expert and its unmodified logit ---

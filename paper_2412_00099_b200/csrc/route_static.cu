@@ -43,6 +43,9 @@ extern "C" int mcce_route_trace_static(const mcce_config* cfg, int32_t n_steps, 
   if (cfg->delta_mode == MCCE_DELTA_FIXED && !fixed_delta) return MCCE_EINVAL;
   if (cfg->hidden_dtype != MCCE_F32 && cfg->hidden_dtype != MCCE_BF16) return MCCE_EINVAL;
   if (hidden && (cfg->d_model < 8 || cfg->d_model % 8)) return MCCE_EINVAL;
+  if (cfg->rerank_mode < MCCE_RERANK_CACHE_PRIOR || cfg->rerank_mode > MCCE_RERANK_CUMSUM) return MCCE_EINVAL;
+  if (cfg->rerank_mode == MCCE_RERANK_MAX_RANK && (cfg->max_rank < 0 || cfg->max_rank > cfg->n_experts))
+    return MCCE_EINVAL;
 
   // layout of the state inside the static array; sizes beyond the array are refused
   const size_t LS = (size_t)cfg->n_layers * cfg->n_streams, E = cfg->n_experts, EW = (E + 31) / 32;
@@ -72,6 +75,7 @@ extern "C" int mcce_route_trace_static(const mcce_config* cfg, int32_t n_steps, 
   p.C = cfg->cache_capacity, p.d = cfg->d_model, p.n_steps = n_steps, p.lambda = cfg->lambda;
   p.delta_mode = cfg->delta_mode, p.renorm = cfg->renorm, p.hidden_bf16 = cfg->hidden_dtype == MCCE_BF16;
   p.n_partials = 1, p.partial_stride = 0;
+  p.rerank_mode = cfg->rerank_mode, p.max_rank = cfg->max_rank, p.cum_threshold = cfg->cum_threshold;
   p.hidden = hidden, p.logits_in = logits_in, p.Wr = Wr, p.fixed_delta = fixed_delta;
   p.stamp = (uint32_t*)(base + o_stamp), p.ever = (uint32_t*)(base + o_ever);
   p.sum_range = (float*)(base + o_sum), p.miss = (uint32_t*)(base + o_miss), p.cold = (uint32_t*)(base + o_cold);

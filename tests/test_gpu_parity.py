@@ -89,6 +89,46 @@ def test_route_from_logits_is_bit_exact(E, K, J, C, lam, dm, renorm, quant, chun
     eng.close()
 
 
+RERANK_CASES = [
+    # mode, E, K, J, C, M, p
+    (1, 8, 2, 1, 4, 0, 0.0),      # Max-Rank with M = 0: nothing promoted
+    (1, 8, 2, 1, 4, 4, 0.0),
+    (1, 60, 4, 2, 30, 12, 0.0),
+    (1, 64, 8, 0, 16, 64, 0.0),   # M = E, J = 0: every cached expert first
+    (1, 130, 7, 2, 40, 33, 0.0),
+    (2, 8, 2, 1, 4, 0, 0.6),      # Cumsum-Threshold
+    (2, 60, 4, 2, 30, 0, 0.5),
+    (2, 64, 6, 2, 24, 0, 0.9),
+    (2, 33, 5, 1, 3, 0, 1.5),     # p > 1: the whole ranking
+    (2, 16, 2, 1, 8, 0, 0.0),     # p = 0: plain top-K
+]
+
+
+@pytest.mark.parametrize("mode,E,K,J,C,M,p", RERANK_CASES)
+def test_baseline_rerankers_match_the_oracle(mode, E, K, J, C, M, p):
+    """Algorithms 1 and 2 as routing modes, identical logits on both sides.  Indices, cache states and
+    counters bit for bit; for the cumulative threshold a step whose partial sum lies within 1e-6 of p
+    may legitimately resolve either way (the probabilities are floating point), which ends the comparison."""
+    L, S, T = 2, 11, 40
+    wl = synth.TINY.with_(L=L, E=E, K=K, J=J, C=C, S=S, d=64, I=64)
+    eng = mb.engine_for(wl, rerank_mode=mode, max_rank=M, cum_threshold=p)
+    o = H.oracle_for(wl, rerank_mode=mode, max_rank=M, cum_threshold=p)
+    z = ar1_logits(E * 7 + mode, T, L, S, E, quant=0.25 if mode == 1 else None)
+    zd = H.to_dev(z)
+    for t in range(T):
+        sel, w = eng.route_step(logits=zd[t:t + 1])
+        osel, ow, margin, _ = o.route(z[t], want_margin=True)
+        same = np.array_equal(sel[0].cpu().numpy(), osel)
+        if not same and mode == 2:
+            bad = np.any(sel[0].cpu().numpy() != osel, axis=-1)
+            assert (margin[bad] < 1e-6).all(), "unexplained difference in the cumulative threshold"
+            print("near-threshold step at token %d: comparison ends" % t)
+            return
+        assert same
+        assert np.allclose(w[0].cpu().numpy(), ow, rtol=1e-5, atol=1e-7)
+    H.assert_state_equal(eng, o)
+
+
 def test_route_initial_state_and_resume():
     wl = synth.TINY.with_(L=2, E=24, K=3, J=1, C=7, S=5, lam=0.5)
     rng = np.random.default_rng(0)
