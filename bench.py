@@ -50,6 +50,7 @@ def parse_args():
                     help="Cache-Prior (Eq. 7, the headline), or the Max-Rank / Cumsum-Threshold baselines")
     ap.add_argument("--max-rank", type=int, default=None, help="M of Max-Rank (default 2K)")
     ap.add_argument("--cum-p", type=float, default=0.5, help="p of Cumsum-Threshold")
+    ap.add_argument("--lifetimes", action="store_true", help="also track and report cache lifetimes")
     ap.add_argument("--impl", default="mcce", choices=["mcce", "reference"])
     ap.add_argument("--ffn", default="auto", choices=["auto", "simt", "tensor"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -205,7 +206,7 @@ def main_arm(args):
     rerank = {"prior": mb.RERANK_CACHE_PRIOR, "maxrank": mb.RERANK_MAX_RANK, "cumsum": mb.RERANK_CUMSUM}[args.rerank]
     max_rank = min(wl.E, args.max_rank if args.max_rank is not None else 2 * wl.K)
     eng = mb.engine_for(wl, ffn_impl=ffn_impl, device=local, rerank_mode=rerank, max_rank=max_rank,
-                        cum_threshold=args.cum_p)
+                        cum_threshold=args.cum_p, track_lifetime=args.lifetimes)
     wdt = torch.bfloat16 if wl.bf16 else torch.float32
 
     # ---- weights, generated on the device ------------------------------------------------------------
@@ -317,6 +318,11 @@ def main_arm(args):
                                      "experts_touched_per_step": touched}),
             "miss_rate": misses / max(1, selections), "roofline": roofline, "kernels": kernels,
             "gpu_launches": int(sum(v[1] for v in prof.values())), "clocks": clocks}
+
+    if args.lifetimes:
+        (n_ev, mean, sd), _ = eng.lifetimes()
+        line["cache_lifetime"] = {"evictions": n_ev, "mean_tokens": mean, "sd_tokens": sd,
+                                  "tokens_per_stream": n_tok}
 
     # ---- end to end through the host-buffer entry point -------------------------------------------------
     if not args.no_e2e:

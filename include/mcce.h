@@ -72,6 +72,7 @@ typedef struct {
   int32_t rerank_mode;    /* MCCE_RERANK_*; lambda / delta_mode only matter for CACHE_PRIOR      */
   int32_t max_rank;       /* M of Algorithm 1, 0..E (MAX_RANK only)                              */
   float cum_threshold;    /* p of Algorithm 2, >= 0 (CUMSUM only)                                */
+  int32_t track_lifetime; /* 1: record how long experts stay cached (mcce_lifetime_stats)         */
 } mcce_config;
 
 typedef struct {
@@ -141,6 +142,15 @@ int mcce_decode_step_host(mcce_ctx* ctx, const void* hidden_host, float* y_host,
 /* Eq. 4 counters, summed over streams: total and per layer (HOST [L], may be NULL).  Synchronises.
  * Also reports MCCE_ETIMEOUT if any kernel of this context gave up on a bounded wait. */
 int mcce_cache_stats(mcce_ctx* ctx, mcce_stats* total /*HOST*/, mcce_stats* per_layer /*HOST*/);
+
+/* Cache lifetimes (the statistic of the paper's Table 2): a lifetime is the number of tokens from the
+ * token that loaded an expert into a (stream, layer) cache to the token that evicted it; experts still
+ * resident are not counted.  total / per_layer (HOST, [L], may be NULL) receive {evictions, sum of
+ * lifetimes, sum of squared lifetimes}; mean = sum/evictions, variance = sumsq/evictions - mean^2.
+ * Needs track_lifetime = 1 in the configuration (MCCE_ESTATE otherwise).  Not part of the state that
+ * mcce_get_cache_state exports.  Synchronises. */
+typedef struct { int64_t evictions, sum, sum_sq; } mcce_lifetime;
+int mcce_lifetime_stats(mcce_ctx* ctx, mcce_lifetime* total /*HOST*/, mcce_lifetime* per_layer /*HOST*/);
 
 /* Canonical cache state: order HOST int32 [L,S,C] most-recently-used first, -1 padded; optional
  * ever HOST uint8 [L,S,E]; delta_sum HOST fp32 [L,S] and *delta_count (optional).  Synchronises. */

@@ -131,7 +131,9 @@ void orc_route_slab(const orc_config* c, const float* z_all /*[L,S,E]*/,
                     int64_t* count_all /*[L,S]*/, int64_t* tok_all /*[L,S]*/,
                     int64_t* counters_all /*[L,S,4]*/, int32_t* sel_all /*[L,S,K]*/,
                     float* w_all /*[L,S,K]*/, float* margin_all /*[L,S] or NULL*/,
-                    float* delta_all /*[L,S] or NULL*/, int s0, int s1) {
+                    float* delta_all /*[L,S] or NULL*/, int64_t* load_tok_all /*[L,S,E] or NULL*/,
+                    int64_t* life_all /*[L,S,3] or NULL: evictions, sum and sum of squares of lifetimes*/,
+                    int s0, int s1) {
   const int L = c->n_layers, E = c->n_experts, K = c->top_k, J = c->top_j, S = c->n_streams;
   const int C = c->cache_capacity;
   for (int l = 0; l < L; ++l) {
@@ -245,6 +247,7 @@ void orc_route_slab(const orc_config* c, const float* z_all /*[L,S,E]*/,
       const int64_t tok = tok_all[p];
       for (int r = 0; r < K; ++r) {
         const int e = sel[order[r]];
+        if (stamp[e] == 0 && load_tok_all) load_tok_all[p * E + e] = tok; /* loaded by this token */
         stamp[e] = (int64_t)E + tok * K + r + 1;
         ever[e] = 1;
       }
@@ -260,6 +263,13 @@ void orc_route_slab(const orc_config* c, const float* z_all /*[L,S,E]*/,
         }
         if (resident <= C) break;
         stamp[victim] = 0;
+        if (life_all) {
+          /* cache lifetime: tokens from the load of an expert to its eviction (Table 2 of the paper) */
+          const int64_t life = tok - load_tok_all[p * E + victim];
+          life_all[p * 3 + 0] += 1;
+          life_all[p * 3 + 1] += life;
+          life_all[p * 3 + 2] += life * life;
+        }
       }
 
       if (delta_all) delta_all[p] = delta;

@@ -99,6 +99,8 @@ class Oracle:
         self.count = np.zeros((L, S), np.int64)
         self.tok = np.zeros((L, S), np.int64)
         self.counters = np.zeros((L, S, 4), np.int64)
+        self.load_tok = np.zeros((L, S, E), np.int64)
+        self.life = np.zeros((L, S, 3), np.int64)
         self.fixed_delta = None if fixed_delta is None else np.ascontiguousarray(fixed_delta, np.float32)
         self.threads = threads
         self._pool = ThreadPoolExecutor(threads) if threads > 1 else None
@@ -113,11 +115,11 @@ class Oracle:
 
     def snapshot(self):
         return tuple(a.copy() for a in (self.stamp, self.ever, self.sum_range, self.count, self.tok,
-                                        self.counters))
+                                        self.counters, self.load_tok, self.life))
 
     def restore(self, snap):
         for dst, src in zip((self.stamp, self.ever, self.sum_range, self.count, self.tok,
-                             self.counters), snap):
+                             self.counters, self.load_tok, self.life), snap):
             dst[...] = src
 
     def reset(self, init_order=None, keep_delta_stats: bool = False):
@@ -126,6 +128,8 @@ class Oracle:
         self.ever[...] = 0
         self.tok[...] = 0
         self.counters[...] = 0
+        self.load_tok[...] = 0
+        self.life[...] = 0
         if not keep_delta_stats:
             self.sum_range[...] = 0
             self.count[...] = 0
@@ -162,7 +166,7 @@ class Oracle:
         self._par(lambda a, b: lib().orc_route_slab(
             C.byref(cc), _p(z), _p(self.fixed_delta), _p(self.stamp), _p(self.ever),
             _p(self.sum_range), _p(self.count), _p(self.tok), _p(self.counters), _p(sel), _p(w),
-            _p(margin), _p(delta), a, b))
+            _p(margin), _p(delta), _p(self.load_tok), _p(self.life), a, b))
         if want_margin:
             return sel, w, margin, delta
         return sel, w
@@ -191,6 +195,14 @@ class Oracle:
                 lib().orc_export_order(_p(self.stamp[l, s]), cfg.n_experts, cfg.cache_capacity,
                                        _p(out[l, s]))
         return out
+
+    def lifetimes(self):
+        """(evictions, mean, standard deviation) of the cache lifetimes of evicted experts, in tokens."""
+        n, s1, s2 = (int(x) for x in self.life.sum(axis=(0, 1)))
+        if n == 0:
+            return 0, 0.0, 0.0
+        mean = s1 / n
+        return n, mean, max(0.0, s2 / n - mean * mean) ** 0.5
 
     def stats(self):
         """{steps, selections, misses, cold_misses} summed over everything, and per layer [L,4]."""

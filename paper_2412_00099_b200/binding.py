@@ -22,7 +22,7 @@ RERANK_CACHE_PRIOR, RERANK_MAX_RANK, RERANK_CUMSUM = 0, 1, 2
 EXPORTS = [
     "mcce_workspace_bytes", "mcce_create", "mcce_destroy", "mcce_set_router", "mcce_set_experts", "mcce_reset",
     "mcce_route_step", "mcce_moe_forward", "mcce_decode_step_host", "mcce_cache_stats", "mcce_get_cache_state",
-    "mcce_get_grouping", "mcce_profile", "mcce_profile_read", "mcce_uses_tensor_path", "mcce_route_trace_static",
+    "mcce_get_grouping", "mcce_lifetime_stats", "mcce_profile", "mcce_profile_read", "mcce_uses_tensor_path", "mcce_route_trace_static",
     "mcce_route_trace_static_limit", "mcce_gen_normal", "mcce_gen_hidden_step", "mcce_gen_philox_words", "mcce_strerror",
     "mcce_last_cuda_error",
 ]
@@ -33,7 +33,8 @@ class Config(C.Structure):
                                          "cache_capacity", "n_streams")] + [
         ("lam", C.c_float), ("delta_mode", C.c_int32), ("renorm", C.c_int32), ("hidden_dtype", C.c_int32),
         ("weight_dtype", C.c_int32), ("ffn_impl", C.c_int32), ("device", C.c_int32),
-        ("rerank_mode", C.c_int32), ("max_rank", C.c_int32), ("cum_threshold", C.c_float)]
+        ("rerank_mode", C.c_int32), ("max_rank", C.c_int32), ("cum_threshold", C.c_float),
+        ("track_lifetime", C.c_int32)]
 
 
 class Stats(C.Structure):
@@ -71,6 +72,7 @@ def load():
         lib.mcce_cache_stats.argtypes = [vp, C.POINTER(Stats), C.POINTER(Stats)]
         lib.mcce_get_cache_state.argtypes = [vp, vp, vp, vp, C.POINTER(C.c_int64)]
         lib.mcce_get_grouping.argtypes = [vp, vp, vp]
+        lib.mcce_lifetime_stats.argtypes = [vp, vp, vp]
         lib.mcce_uses_tensor_path.argtypes = [vp]
         lib.mcce_route_trace_static_limit.restype = C.c_size_t
         lib.mcce_route_trace_static.argtypes = [C.POINTER(Config), i32, vp, vp, vp, vp, vp, vp, C.POINTER(Stats), vp]
@@ -116,12 +118,13 @@ class Engine:
     """One mcce context: the cache state of every (stream, layer) plus borrowed weights."""
 
     def __init__(self, *, L, E, K, J, n_shared, d, I, C_cap, S, lam, delta_mode=DELTA_RUNNING, renorm=1, dtype=BF16,
-                 ffn_impl=FFN_AUTO, device=0, rerank_mode=RERANK_CACHE_PRIOR, max_rank=0, cum_threshold=0.0):
+                 ffn_impl=FFN_AUTO, device=0, rerank_mode=RERANK_CACHE_PRIOR, max_rank=0, cum_threshold=0.0,
+                 track_lifetime=False):
         if not torch.cuda.is_available():
             raise McceError("no CUDA device: this library has no CPU path")
         self.lib = load()
         self.cfg = Config(L, E, K, J, n_shared, d, I, C_cap, S, lam, delta_mode, renorm, dtype, dtype, ffn_impl,
-                          device, rerank_mode, max_rank, cum_threshold)
+                          device, rerank_mode, max_rank, cum_threshold, int(track_lifetime))
         self.device = torch.device("cuda", device)
         nbytes = self.lib.mcce_workspace_bytes(C.byref(self.cfg))
         if nbytes == 0:
@@ -231,6 +234,16 @@ class Engine:
         n = np.zeros(len(self.KERNELS), np.int64)
         _check(self.lib.mcce_profile_read(self.ctx, _ptr(ms), _ptr(n), int(reset)), self.ctx)
         return {k: (float(ms[i]), int(n[i])) for i, k in enumerate(self.KERNELS)}
+
+    def lifetimes(self):
+        """(evictions, mean, standard deviation) of cache lifetimes in tokens, and the raw per-layer sums."""
+        total = np.zeros(3, np.int64)
+        per = np.zeros((self.L, 3), np.int64)
+        _check(self.lib.mcce_lifetime_stats(self.ctx, _ptr(total), _ptr(per)), self.ctx)
+        n, s1, s2 = (int(x) for x in total)
+        mean = s1 / n if n else 0.0
+        sd = max(0.0, s2 / n - mean * mean) ** 0.5 if n else 0.0
+        return (n, mean, sd), per
 
     def grouping(self):
         offsets = np.empty((self.L, self.E + 1), np.int32)

@@ -18,7 +18,8 @@ struct mcce_ctx {
   int EW;
   size_t rows;  // rows of H / O: L*S*K routed pairs + L*n_sh*S shared
   // workspace pieces (device)
-  uint32_t *stamp, *ever, *miss, *cold, *err;
+  uint32_t *stamp, *ever, *miss, *cold, *err, *load_tok;
+  unsigned long long* life;
   float* sum_range;
   unsigned long long* stats_dev;
   int32_t *offsets, *perm, *inv;
@@ -71,12 +72,13 @@ bool valid(const mcce_config* c) {
   if (c->rerank_mode < MCCE_RERANK_CACHE_PRIOR || c->rerank_mode > MCCE_RERANK_CUMSUM) return false;
   if (c->rerank_mode == MCCE_RERANK_MAX_RANK && (c->max_rank < 0 || c->max_rank > c->n_experts)) return false;
   if (c->rerank_mode == MCCE_RERANK_CUMSUM && !(c->cum_threshold >= 0.f)) return false;
+  if (c->track_lifetime != 0 && c->track_lifetime != 1) return false;
   return true;
 }
 
 struct Layout {
   size_t stamp, ever, sum_range, miss, cold, err, stats, offsets, perm, inv, Xg, H, O, st_hidden, st_sel, st_w, st_y,
-      wr_terms, z_buf, total;
+      wr_terms, z_buf, load_tok, life, total;
 };
 
 Layout layout_of(const mcce_config& c) {
@@ -110,6 +112,8 @@ Layout layout_of(const mcce_config& c) {
   const bool rg = router_gemm_applicable(c);
   o.wr_terms = take(rg ? 3 * L * E * d * 2 : 0);
   o.z_buf = take(rg ? (size_t)router_gemm_steps_max() * L * S * E * 4 : 0);
+  o.load_tok = take(c.track_lifetime ? L * S * E * 4 : 0);
+  o.life = take(c.track_lifetime ? L * S * 3 * 8 : 0);
   o.total = p;
   return o;
 }
@@ -202,9 +206,12 @@ extern "C" int mcce_create(const mcce_config* cfg, void* workspace, size_t works
   ctx->use_tc = cfg->ffn_impl != MCCE_FFN_SIMT && tc_applicable(*cfg);
   ctx->use_tc_router = router_gemm_applicable(*cfg);
   ctx->wr_terms = w + lo.wr_terms, ctx->z_buf = (float*)(w + lo.z_buf);
+  ctx->load_tok = cfg->track_lifetime ? (uint32_t*)(w + lo.load_tok) : nullptr;
+  ctx->life = cfg->track_lifetime ? (unsigned long long*)(w + lo.life) : nullptr;
   cudaError_t e = cudaSetDevice(cfg->device);
   // state arrays and the activation buffers start at zero (the slack rows must hold finite values)
   if (e == cudaSuccess) e = cudaMemset(w, 0, lo.O);
+  if (e == cudaSuccess && cfg->track_lifetime) e = cudaMemset(w + lo.load_tok, 0, lo.total - lo.load_tok);
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
   if (e != cudaSuccess) {
     delete ctx;
@@ -280,6 +287,10 @@ extern "C" int mcce_reset(mcce_ctx* ctx, const int32_t* init_order, int keep_del
   CK(cudaMemset(ctx->miss, 0, LS * 4));
   CK(cudaMemset(ctx->cold, 0, LS * 4));
   CK(cudaMemset(ctx->err, 0, 64));
+  if (ctx->load_tok) {
+    CK(cudaMemset(ctx->load_tok, 0, LS * E * 4));
+    CK(cudaMemset(ctx->life, 0, LS * 3 * 8));
+  }
   if (delta_sum) {
     CK(cudaMemcpy(ctx->sum_range, delta_sum, LS * 4, cudaMemcpyHostToDevice));
     ctx->delta_cnt = (uint64_t)delta_count;
@@ -311,6 +322,7 @@ extern "C" int mcce_route_step(mcce_ctx* ctx, int32_t n_steps, const void* hidde
   p.hidden_bf16 = c.hidden_dtype == MCCE_BF16;
   p.Wr = ctx->Wr, p.fixed_delta = ctx->fixed_delta;
   p.stamp = ctx->stamp, p.ever = ctx->ever, p.sum_range = ctx->sum_range, p.miss = ctx->miss, p.cold = ctx->cold;
+  p.load_tok = ctx->load_tok, p.life = ctx->life;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   if (hidden && ctx->use_tc_router && ctx->rg.ready) {
     // logits by the tensor-core GEMM, a few tokens at a time, then the fused tail on those logits
@@ -436,6 +448,27 @@ extern "C" int mcce_get_cache_state(mcce_ctx* ctx, int32_t* order, uint8_t* ever
   return MCCE_OK;
 }
 
+extern "C" int mcce_lifetime_stats(mcce_ctx* ctx, mcce_lifetime* total, mcce_lifetime* per_layer) {
+  if (!ctx || !total) return MCCE_EINVAL;
+  if (!ctx->life) return MCCE_ESTATE;
+  const mcce_config& c = ctx->cfg;
+  CK(cudaSetDevice(c.device));
+  CK(cudaDeviceSynchronize());
+  std::vector<unsigned long long> h((size_t)c.n_layers * c.n_streams * 3);
+  CK(cudaMemcpy(h.data(), ctx->life, h.size() * 8, cudaMemcpyDeviceToHost));
+  memset(total, 0, sizeof(*total));
+  for (int l = 0; l < c.n_layers; ++l) {
+    mcce_lifetime s = {0, 0, 0};
+    for (int q = 0; q < c.n_streams; ++q) {
+      const unsigned long long* r = &h[((size_t)l * c.n_streams + q) * 3];
+      s.evictions += (int64_t)r[0], s.sum += (int64_t)r[1], s.sum_sq += (int64_t)r[2];
+    }
+    if (per_layer) per_layer[l] = s;
+    total->evictions += s.evictions, total->sum += s.sum, total->sum_sq += s.sum_sq;
+  }
+  return MCCE_OK;
+}
+
 extern "C" int mcce_get_grouping(mcce_ctx* ctx, int32_t* offsets, int32_t* perm) {
   if (!ctx || !offsets || !perm) return MCCE_EINVAL;
   const mcce_config& c = ctx->cfg;
@@ -486,7 +519,9 @@ extern "C" const char* mcce_strerror(int code) {
     case MCCE_OK: return "ok";
     case MCCE_EINVAL: return "invalid argument or unsupported configuration";
     case MCCE_ENOSPC: return "workspace too small";
-    case MCCE_ESTATE: return "weights not set, or a 32-bit recency counter would overflow (call mcce_reset)";
+    case MCCE_ESTATE:
+      return "weights not set, a feature not enabled in the configuration, or a 32-bit recency counter would "
+             "overflow (call mcce_reset)";
     case MCCE_ECUDA: return "CUDA call failed (see mcce_last_cuda_error)";
     case MCCE_ETIMEOUT: return "a bounded wait inside a kernel gave up";
     case MCCE_ELIMIT:

@@ -33,6 +33,8 @@ struct RouteParams {
   float* sum_range;          // [L,S]
   uint32_t* miss;            // [L,S]
   uint32_t* cold;            // [L,S]
+  uint32_t* load_tok;        // [L,S,E] token that loaded each resident expert, or null (lifetimes not tracked)
+  unsigned long long* life;  // [L,S,3]  evictions, sum and sum of squares of cache lifetimes
   int32_t* sel_idx;          // [n_steps,L,S,K]
   float* sel_w;              // [n_steps,L,S,K]
   float* logits_out;         // [n_steps,L,S,E] or null

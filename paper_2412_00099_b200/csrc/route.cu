@@ -65,6 +65,9 @@ __global__ void __launch_bounds__(kWarps * 32) route_kernel(const RouteParams p,
 
   // ---- state of this (layer, stream) into registers -------------------------------------------
   uint32_t st[NE];
+  uint32_t ld[NE];   // token that loaded each resident expert (only when lifetimes are tracked)
+  unsigned long long life_n = 0ull, life_sum = 0ull, life_sq = 0ull;
+  const bool track = p.load_tok != nullptr;
   uint32_t everb = 0u;
   float sum_range = 0.f;
   uint32_t miss_c = 0u, cold_c = 0u;
@@ -73,6 +76,7 @@ __global__ void __launch_bounds__(kWarps * 32) route_kernel(const RouteParams p,
     for (int i = 0; i < NE; ++i) {
       const int e = lane + 32 * i;
       st[i] = e < E ? p.stamp[pair * E + e] : 0u;
+      ld[i] = (track && e < E) ? p.load_tok[pair * E + e] : 0u;
       if (i < EW) everb |= ((p.ever[pair * EW + i] >> lane) & 1u) << i;
     }
     sum_range = p.sum_range[pair];
@@ -80,7 +84,7 @@ __global__ void __launch_bounds__(kWarps * 32) route_kernel(const RouteParams p,
     cold_c = p.cold[pair];
   } else {
 #pragma unroll
-    for (int i = 0; i < NE; ++i) st[i] = 0u;
+    for (int i = 0; i < NE; ++i) st[i] = ld[i] = 0u;
   }
 
   for (int t = 0; t < p.n_steps; ++t) {
@@ -306,7 +310,10 @@ __global__ void __launch_bounds__(kWarps * 32) route_kernel(const RouteParams p,
         const int slot = eo >> 5;
 #pragma unroll
         for (int i = 0; i < NE; ++i)
-          if (i == slot) st[i] = base + (uint32_t)po;
+          if (i == slot) {
+            if (st[i] == 0u) ld[i] = p.tok0 + (uint32_t)t;   // a miss: loaded by this token
+            st[i] = base + (uint32_t)po;
+          }
         everb |= 1u << slot;
       }
     }
@@ -322,7 +329,13 @@ __global__ void __launch_bounds__(kWarps * 32) route_kernel(const RouteParams p,
       const uint32_t m = __reduce_min_sync(kFull, lmin);
 #pragma unroll
       for (int i = 0; i < NE; ++i)
-        if (st[i] == m) st[i] = 0u;
+        if (st[i] == m) {
+          st[i] = 0u;
+          if (track) {   // cache lifetime of the evicted expert, in tokens (Table 2 of the paper)
+            const unsigned long long life = (unsigned long long)(p.tok0 + (uint32_t)t - ld[i]);
+            life_n += 1ull, life_sum += life, life_sq += life * life;
+          }
+        }
       --resident;
     }
 
@@ -338,9 +351,22 @@ __global__ void __launch_bounds__(kWarps * 32) route_kernel(const RouteParams p,
     for (int i = 0; i < NE; ++i) {
       const int e = lane + 32 * i;
       if (e < E) p.stamp[pair * E + e] = st[i];
+      if (track && e < E) p.load_tok[pair * E + e] = ld[i];
       if (i < EW) {
         const uint32_t word = __ballot_sync(kFull, (everb >> i) & 1u);
         if (lane == 0) p.ever[pair * EW + i] = word;
+      }
+    }
+    if (track) {
+      for (int o = 16; o > 0; o >>= 1) {
+        life_n += __shfl_xor_sync(kFull, life_n, o);
+        life_sum += __shfl_xor_sync(kFull, life_sum, o);
+        life_sq += __shfl_xor_sync(kFull, life_sq, o);
+      }
+      if (lane == 0) {
+        p.life[pair * 3 + 0] += life_n;
+        p.life[pair * 3 + 1] += life_sum;
+        p.life[pair * 3 + 2] += life_sq;
       }
     }
     if (lane == 0) {

@@ -41,6 +41,8 @@ def assert_state_equal(eng, o):
     ot, opl = o.stats()
     assert list(total) == ot.tolist()
     assert [list(p) for p in per_layer] == opl.tolist()
+    if eng.cfg.track_lifetime:
+        assert eng.lifetimes()[1].tolist() == o.life.sum(axis=1).tolist()
 
 
 def check_route_exact(eng, o, z_all: np.ndarray, chunk: int = 1, check_every: int = 8):

@@ -80,7 +80,7 @@ def test_route_from_logits_is_bit_exact(E, K, J, C, lam, dm, renorm, quant, chun
     L, S, T = 3, 19, 48          # S not a multiple of the CTA's stream block
     wl = synth.TINY.with_(L=L, E=E, K=K, J=J, C=C, S=S, lam=lam, d=64, I=64)
     fixed = np.linspace(2.0, 4.0, L).astype(np.float32) if dm else None
-    eng = mb.engine_for(wl, delta_mode=dm, renorm=renorm)
+    eng = mb.engine_for(wl, delta_mode=dm, renorm=renorm, track_lifetime=True)
     if dm:
         eng.set_router(torch.zeros((L, E, 64), device="cuda"), H.to_dev(fixed))
     o = H.oracle_for(wl, delta_mode=dm, renorm=renorm, fixed_delta=fixed)
@@ -111,7 +111,7 @@ def test_baseline_rerankers_match_the_oracle(mode, E, K, J, C, M, p):
     may legitimately resolve either way (the probabilities are floating point), which ends the comparison."""
     L, S, T = 2, 11, 40
     wl = synth.TINY.with_(L=L, E=E, K=K, J=J, C=C, S=S, d=64, I=64)
-    eng = mb.engine_for(wl, rerank_mode=mode, max_rank=M, cum_threshold=p)
+    eng = mb.engine_for(wl, rerank_mode=mode, max_rank=M, cum_threshold=p, track_lifetime=True)
     o = H.oracle_for(wl, rerank_mode=mode, max_rank=M, cum_threshold=p)
     z = ar1_logits(E * 7 + mode, T, L, S, E, quant=0.25 if mode == 1 else None)
     zd = H.to_dev(z)

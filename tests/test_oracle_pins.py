@@ -557,3 +557,41 @@ def make_and_run_plain(E, K, J, C, seed):
     for z in ar1_logits(rng, 60, 1, 3, E):
         o.route(z)
     return o.stats()[0][2]
+
+
+# ---- cache lifetimes (the statistic of the paper's Table 2) -------------------------------------------
+def test_lifetimes_match_brute_force_over_resident_sets():
+    """Lifetime of a residency = number of tokens from the token that loaded the expert to the token
+    that evicted it; recomputed here from the exported resident set after every token."""
+    rng = np.random.default_rng(53)
+    for (E, K, J, C, lam) in [(8, 2, 1, 4, 0.0), (8, 2, 1, 4, 0.7), (10, 3, 0, 2, 0.3), (6, 2, 1, 1, 0.5)]:
+        o = make(E=E, K=K, J=J, C=C, lam=lam, L=1, S=2)
+        loaded = [dict(), dict()]
+        lives = []
+        for t, z in enumerate(ar1_logits(rng, 120, 1, 2, E, rho=0.6)):
+            sel, _ = o.route(z)
+            after = o.order()
+            for s in range(2):
+                now = set(e for e in after[0, s].tolist() if e >= 0)
+                for e in sel[0, s].tolist():                 # every selected expert is (re)loaded if absent
+                    loaded[s].setdefault(e, t)
+                for e in list(loaded[s]):
+                    if e not in now:                          # evicted during this token
+                        lives.append(t - loaded[s].pop(e))
+        n, mean, sd = o.lifetimes()
+        assert n == len(lives)
+        assert mean == pytest.approx(np.mean(lives)) and sd == pytest.approx(np.std(lives))
+
+
+def test_lifetimes_grow_with_lambda_on_tiny():
+    """Direction of Table 2: experts stay resident longer under cache-aware routing."""
+    wl = synth.TINY
+    Wr = wl.router()
+    xs = list(wl.hidden_trace(wl.T))
+    means = []
+    for lam in (0.0, 0.5):
+        o = orc.Oracle(orc.OracleConfig(wl.L, wl.E, wl.K, 0, 0, wl.d, wl.I, wl.C, wl.S, lam, 0, 1, 0))
+        for x in xs:
+            o.route(o.logits(Wr, x))
+        means.append(o.lifetimes()[1])
+    assert means[1] > 1.5 * means[0]
