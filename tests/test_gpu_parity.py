@@ -129,6 +129,16 @@ def test_baseline_rerankers_match_the_oracle(mode, E, K, J, C, M, p):
     H.assert_state_equal(eng, o)
 
 
+def test_cumsum_threshold_reached_exactly_on_gpu():
+    """Four equal logits: probabilities of exactly 1/4; p = 1/2 stops after two ranks (see the oracle pin)."""
+    for p, want in ((0.5, 0), (0.51, 2)):
+        eng = mb.Engine(L=1, E=4, K=1, J=0, n_shared=0, d=64, I=64, C_cap=2, S=1, lam=0.5, dtype=mb.F32,
+                        rerank_mode=mb.RERANK_CUMSUM, cum_threshold=p)
+        eng.reset(init_order=np.array([[[2, -1]]], np.int32))
+        sel, _ = eng.route_step(logits=torch.zeros((1, 1, 1, 4), device="cuda"))
+        assert sel.flatten().tolist() == [want]
+
+
 def test_route_initial_state_and_resume():
     wl = synth.TINY.with_(L=2, E=24, K=3, J=1, C=7, S=5, lam=0.5)
     rng = np.random.default_rng(0)

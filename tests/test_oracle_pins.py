@@ -139,6 +139,27 @@ def test_cumsum_threshold_picks_smallest_M():
     assert M == 4 and out == [1, 3, 4, 2, 5, 6]
     M, out = orc.cumsum_threshold(r, w, in_cache, 0.3, 0)
     assert M == 1 and out == r                          # peaky router: nothing may be promoted
+    # "until the threshold is reached": a partial sum that equals p exactly stops the walk
+    w2 = np.array([0.0, 0.5, 0.25, 0.125, 0.0625, 0.03125, 0.03125], np.float32)
+    M, out = orc.cumsum_threshold(r, w2, in_cache, 0.75, 0)
+    assert M == 2 and out == r
+    M, out = orc.cumsum_threshold(r, w2, in_cache, 0.875, 0)
+    assert M == 3 and out == [3, 1, 2, 4, 5, 6]
+
+
+def test_cumsum_mode_reaches_the_threshold_exactly():
+    """Four equal logits give probabilities of exactly 1/4: with p = 1/2 the walk stops after two ranks, so
+    the cached expert at rank 3 is outside the window and the router's top-1 stays selected."""
+    cfg = orc.OracleConfig(1, 4, 1, 0, 0, 16, 8, 2, 1, 0.5, 0, 1, 0, 2, 0, 0.5)
+    o = orc.Oracle(cfg)
+    o.reset(init_order=np.array([[[2, -1]]], np.int32))
+    sel, _ = o.route(np.zeros((1, 1, 4), np.float32))
+    assert sel[0, 0].tolist() == [0]
+    cfg.cum_threshold = 0.51                    # now three ranks are needed and the cached expert wins
+    o = orc.Oracle(cfg)
+    o.reset(init_order=np.array([[[2, -1]]], np.int32))
+    sel, _ = o.route(np.zeros((1, 1, 4), np.float32))
+    assert sel[0, 0].tolist() == [2]
 
 
 # ---- hand-computed instances of Eq. 7 / Eq. 8 / Eq. 4 / the in-token LRU order --------------------
