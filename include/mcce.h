@@ -222,6 +222,13 @@ int mcce_route_trace_static(const mcce_config* cfg /*HOST*/, int32_t n_steps, co
                             const float* logits_in, const float* fixed_delta, int32_t* sel_idx, float* sel_w,
                             mcce_stats* totals_host, void* cuda_stream);
 
+/* Self-test of the bounded waits that the tensor-core kernels use (no counterpart in the paper).  Launches
+ * a one-CTA kernel that waits on a barrier nothing ever arrives at, with a limit of limit_ns (1..1e9).  The
+ * wait must give up and the kernel must return: MCCE_OK then, and the context's error word is set, so that
+ * the next mcce_cache_stats reports MCCE_ETIMEOUT until mcce_reset clears it.  The GPU context stays usable.
+ * Synchronises. */
+int mcce_selftest_wait_timeout(mcce_ctx* ctx, uint64_t limit_ns);
+
 /* 1 if mcce_moe_forward of this context runs the tcgen05/TMA expert kernels, 0 if the fp32-pipe ones. */
 int mcce_uses_tensor_path(const mcce_ctx* ctx);
 

@@ -22,7 +22,7 @@ RERANK_CACHE_PRIOR, RERANK_MAX_RANK, RERANK_CUMSUM = 0, 1, 2
 EXPORTS = [
     "mcce_workspace_bytes", "mcce_create", "mcce_destroy", "mcce_set_router", "mcce_set_experts", "mcce_reset",
     "mcce_route_step", "mcce_moe_forward", "mcce_decode_step_host", "mcce_cache_stats", "mcce_get_cache_state",
-    "mcce_get_grouping", "mcce_lifetime_stats", "mcce_profile", "mcce_profile_read", "mcce_uses_tensor_path", "mcce_route_trace_static",
+    "mcce_get_grouping", "mcce_lifetime_stats", "mcce_profile", "mcce_profile_read", "mcce_uses_tensor_path", "mcce_selftest_wait_timeout", "mcce_route_trace_static",
     "mcce_route_trace_static_limit", "mcce_gen_normal", "mcce_gen_hidden_step", "mcce_gen_philox_words", "mcce_strerror",
     "mcce_last_cuda_error",
 ]
@@ -74,6 +74,7 @@ def load():
         lib.mcce_get_grouping.argtypes = [vp, vp, vp]
         lib.mcce_lifetime_stats.argtypes = [vp, vp, vp]
         lib.mcce_uses_tensor_path.argtypes = [vp]
+        lib.mcce_selftest_wait_timeout.argtypes = [vp, C.c_uint64]
         lib.mcce_route_trace_static_limit.restype = C.c_size_t
         lib.mcce_route_trace_static.argtypes = [C.POINTER(Config), i32, vp, vp, vp, vp, vp, vp, C.POINTER(Stats), vp]
         lib.mcce_profile.argtypes = [vp, C.c_int]

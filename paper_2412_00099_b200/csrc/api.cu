@@ -479,6 +479,18 @@ extern "C" int mcce_get_grouping(mcce_ctx* ctx, int32_t* offsets, int32_t* perm)
   return MCCE_OK;
 }
 
+extern "C" int mcce_selftest_wait_timeout(mcce_ctx* ctx, uint64_t limit_ns) {
+  if (!ctx || limit_ns == 0 || limit_ns > 1000000000ull) return MCCE_EINVAL;
+  CK(cudaSetDevice(ctx->cfg.device));
+  uint32_t* outcome = ctx->err + 8;   // a spare word of the error block
+  CK(cudaMemset(outcome, 0, 4));
+  CK(launch_wait_timeout_selftest(ctx->err, limit_ns, outcome, 0));
+  CK(cudaDeviceSynchronize());
+  uint32_t h = 0;
+  CK(cudaMemcpy(&h, outcome, 4, cudaMemcpyDeviceToHost));
+  return h == 2u ? MCCE_OK : MCCE_ESTATE;
+}
+
 extern "C" int mcce_uses_tensor_path(const mcce_ctx* ctx) { return ctx ? ctx->use_tc : MCCE_EINVAL; }
 
 extern "C" int mcce_profile(mcce_ctx* ctx, int enable) {

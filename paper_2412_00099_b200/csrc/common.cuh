@@ -80,6 +80,8 @@ int router_gemm_plan(const mcce_config& c, const float* Wr, void* terms, RouterG
 cudaError_t router_gemm_launch(RouterGemmPlan& plan, const mcce_config& c, const void* hidden, int n_steps, float* Z,
                                int* k_split, uint32_t* err, cudaStream_t st);
 
+cudaError_t launch_wait_timeout_selftest(uint32_t* err, unsigned long long limit_ns, uint32_t* outcome,
+                                         cudaStream_t st);
 cudaError_t launch_route(const RouteParams& p, cudaStream_t st);
 cudaError_t launch_group(const GroupParams& p, cudaStream_t st);
 cudaError_t launch_gather(const FfnParams& p, cudaStream_t st);

@@ -236,6 +236,22 @@ router_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs a) {
   if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
 }
 
+// Self-test of the bounded wait: one CTA waits on an mbarrier that nothing will ever arrive at; the wait
+// must give up after limit_ns, record the error word and let the kernel return normally.
+__global__ void wait_timeout_selftest_kernel(uint32_t* err, unsigned long long limit_ns, uint32_t* outcome) {
+  __shared__ uint64_t bar;
+  __shared__ uint32_t abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    abort_flag = 0u;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  const bool ok = mbar_wait(smem_u32(&bar), 0u, &abort_flag, err, 99u, limit_ns);
+  __syncthreads();
+  if (threadIdx.x == 0) *outcome = ok ? 1u : 2u;   // 2: the wait gave up, as it must
+}
+
 // W (fp32) -> hi, mid, lo (bf16): each term is the bf16 rounding of what the earlier terms left over.
 __global__ void split_router_kernel(const float* W, __nv_bfloat16* out, size_t n) {
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
@@ -254,6 +270,12 @@ __global__ void split_router_kernel(const float* W, __nv_bfloat16* out, size_t n
 
 // Router rows loaded per term tile: all 128 of a full tile, else E rounded up to the 8-row swizzle group.
 static int term_rows(int E) { return E >= kTileM ? kTileM : (E + 7) & ~7; }
+
+cudaError_t launch_wait_timeout_selftest(uint32_t* err, unsigned long long limit_ns, uint32_t* outcome,
+                                         cudaStream_t st) {
+  wait_timeout_selftest_kernel<<<1, 64, 0, st>>>(err, limit_ns, outcome);
+  return cudaGetLastError();
+}
 
 bool router_gemm_applicable(const mcce_config& c) { return c.hidden_dtype == MCCE_BF16 && c.d_model % kTileK == 0; }
 

@@ -40,14 +40,15 @@ __device__ __forceinline__ unsigned long long global_ns() {
 
 // Bounded wait.  Returns false if the CTA is aborting (this wait timed out, or another one did).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                          uint32_t* err, uint32_t code) {
+                                          uint32_t* err, uint32_t code,
+                                          unsigned long long limit_ns = kWaitLimitNs) {
   if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = global_ns();
   for (uint32_t it = 1;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((it & 255u) == 0u) {
       if (*abort_flag) return false;
-      if (global_ns() - t0 > kWaitLimitNs) {
+      if (global_ns() - t0 > limit_ns) {
         *abort_flag = 1u;
         atomicCAS(err, 0u, code);
         return false;

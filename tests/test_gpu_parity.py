@@ -325,6 +325,19 @@ def test_decode_step_from_host_buffers():
         assert torch.allclose(yh, y.cpu(), rtol=1e-5, atol=1e-6)
 
 
+def test_bounded_wait_gives_up_and_the_context_survives():
+    """A wait that can never be satisfied ends after its limit with an error status instead of hanging;
+    afterwards the same context routes correctly."""
+    wl = synth.TINY.with_(L=1, S=4)
+    eng = mb.engine_for(wl)
+    assert eng.lib.mcce_selftest_wait_timeout(eng.ctx, 1_000_000) == 0          # 1 ms limit
+    with pytest.raises(mb.McceError, match="bounded wait"):
+        eng.cache_stats()
+    eng.reset()                                                                  # clears the error word
+    z = ar1_logits(5, 4, wl.L, wl.S, wl.E)
+    H.check_route_exact(eng, H.oracle_for(wl), z)
+
+
 # ---- argument checking: errors come back as codes, nothing is launched ------------------------------------
 def test_bad_arguments_are_rejected():
     with pytest.raises(mb.McceError):
