@@ -285,15 +285,20 @@ def test_model_shaped_forward_tensor_core_bf16(base, kw):
     print("%s tensor-core forward: max abs err %.2e" % (base.name, worst[0]))
 
 
-def test_tensor_core_path_agrees_with_simt_path():
-    """Same inputs through both expert-FFN implementations of the library (a consistency check on
-    top of the oracle comparisons above)."""
-    wl = synth.QWEN.with_(L=2, S=64, E=20, K=4, C=10, d=512, I=640, n_shared=1)
+@pytest.mark.parametrize("skew", [False, True])
+def test_tensor_core_path_agrees_with_simt_path(skew):
+    """Same inputs through both expert-FFN implementations of the library (a consistency check on top of
+    the oracle comparisons above).  With skew every stream selects expert 0 as well, so that one group is
+    several times larger than the token tile the launch was sized for and takes several passes."""
+    wl = synth.QWEN.with_(L=2, S=72, E=20, K=4, C=10, d=512, I=640, n_shared=1)
     W = {k: (None if v is None else H.to_dev(v)) for k, v in H.weights_for(wl).items()}
     x = H.to_dev(next(iter(wl.hidden_trace(1))))
     rng = np.random.default_rng(1)
-    sel = H.to_dev(np.stack([[rng.choice(wl.E, wl.K, replace=False) for _ in range(wl.S)]
-                             for _ in range(wl.L)]).astype(np.int32))
+    sel = np.stack([[rng.choice(np.arange(1, wl.E), wl.K, replace=False) for _ in range(wl.S)]
+                    for _ in range(wl.L)]).astype(np.int32)
+    if skew:
+        sel[..., 0] = 0
+    sel = H.to_dev(sel)
     w = torch.rand((wl.L, wl.S, wl.K), device="cuda")
     ys = []
     for impl in (mb.FFN_SIMT, mb.FFN_TENSOR):
