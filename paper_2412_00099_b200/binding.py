@@ -12,7 +12,8 @@ import numpy as np
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libmcce.so")
+# MCCE_LIB in the environment points at another build of the library (e.g. to compare two versions)
+LIB_PATH = os.environ.get("MCCE_LIB") or os.path.join(_HERE, "libmcce.so")
 
 F32, BF16 = 0, 1
 DELTA_RUNNING, DELTA_FIXED = 0, 1

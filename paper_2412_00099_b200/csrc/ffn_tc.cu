@@ -37,10 +37,14 @@ constexpr uint32_t kBBytes = kNMax * kTileK * 2;    // 16 KB
 
 template <bool UP>
 struct Cfg {
-  static constexpr int kStages = UP ? 4 : 7;
-  static constexpr uint32_t kStageBytes = (UP ? 2 : 1) * kABytes + kBBytes;
-  static constexpr int kAccCols = UP ? 2 * kNMax : kNMax;   // TMEM columns per accumulator buffer
-  static constexpr int kTmemCols = 2 * kAccCols;            // two buffers: 512 / 256
+  // Both kernels stream TWO 128-row weight tiles per stage against one tile of token rows: gate and up
+  // rows of the same range (up), or two consecutive row ranges of W_d (down).  The token rows come
+  // from L2 but still count against what an SM can take in per microsecond, so sharing them between
+  // two weight tiles is worth 10 % on the down kernel.
+  static constexpr int kStages = 4;
+  static constexpr uint32_t kStageBytes = 2 * kABytes + kBBytes;
+  static constexpr int kAccCols = 2 * kNMax;                // TMEM columns per accumulator buffer
+  static constexpr int kTmemCols = 2 * kAccCols;            // two buffers: 512
   static constexpr size_t kSmemBytes = (size_t)kStages * kStageBytes + 1024 /*align*/ + 256 /*barriers*/;
 };
 
@@ -72,6 +76,7 @@ struct Item {
   size_t orow;    // first row in H / O
   int col0;       // first output column (= weight row inside the expert) of this tile
   int l;          // layer
+  int ntile;      // weight tiles in this item: 2, or 1 for the last odd row range of the down kernel
   bool shared;
 };
 
@@ -82,14 +87,15 @@ __host__ __device__ __forceinline__ int items_per_layer(int E, int n_sh, int S, 
 template <bool UP>
 __device__ __forceinline__ Item decode(const TcArgs& a, int w) {
   const int rows = UP ? a.I : a.d;
-  const int RT = rows / kTileM, P = a.S * a.K, NC = (a.S + kNMax - 1) / kNMax;
+  const int span = UP ? kTileM : 2 * kTileM;   // output features covered by one item
+  const int RT = (rows + span - 1) / span, P = a.S * a.K, NC = (a.S + kNMax - 1) / kNMax;
   const int per_layer = items_per_layer(a.E, a.n_sh, a.S, RT);
   const int l = w / per_layer, wl = w % per_layer;
   Item it;
   it.l = l;
   if (wl < a.E * RT) {
     const int g = wl / RT;
-    it.col0 = (wl % RT) * kTileM;
+    it.col0 = (wl % RT) * span;
     const int o0 = __ldg(a.offsets + (size_t)l * (a.E + 1) + g);
     it.m = __ldg(a.offsets + (size_t)l * (a.E + 1) + g + 1) - o0;
     it.shared = false;
@@ -99,13 +105,14 @@ __device__ __forceinline__ Item decode(const TcArgs& a, int w) {
   } else {
     const int idx = wl - a.E * RT;
     const int c = idx % NC, rt = (idx / NC) % RT, q = idx / (NC * RT);
-    it.col0 = rt * kTileM;
+    it.col0 = rt * span;
     it.m = min(kNMax, a.S - c * kNMax);
     it.shared = true;
     it.wrow = (l * a.n_sh + q) * rows + it.col0;
     it.orow = (size_t)a.L * P + (size_t)(l * a.n_sh + q) * a.S + c * kNMax;
     it.xrow = UP ? l * a.S + c * kNMax : (int)it.orow;   // up: rows of the hidden tensor; down: rows of H
   }
+  it.ntile = (UP || it.col0 + 2 * kTileM <= rows) ? 2 : 1;
   return it;
 }
 
@@ -159,7 +166,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, const TcArgs a) {
         const CUtensorMap* mx = it.shared ? &maps.xs : &maps.x;
         for (int c0 = 0; c0 < it.m && alive; c0 += kNMax) {
           const int n = (min(kNMax, it.m - c0) + 15) & ~15;
-          const uint32_t tx = (UP ? 2 : 1) * kABytes + (uint32_t)n * kTileK * 2;
+          const uint32_t tx = (uint32_t)it.ntile * kABytes + (uint32_t)n * kTileK * 2;
           for (int kt = 0; kt < KT; ++kt) {
             if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, a.err, 1u)) {
               alive = false;
@@ -170,7 +177,8 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, const TcArgs a) {
             mbar_expect_tx(full, tx);
             tma_load_2d(sa, mw0, kt * kTileK, it.wrow, full);
             if (UP) tma_load_2d(sa + kABytes, mw1, kt * kTileK, it.wrow, full);
-            const uint32_t sb = sa + (UP ? 2 : 1) * kABytes;
+            else if (it.ntile == 2) tma_load_2d(sa + kABytes, mw0, kt * kTileK, it.wrow + kTileM, full);
+            const uint32_t sb = sa + 2 * kABytes;
             for (int j = 0; j < n; j += kXBox)
               tma_load_2d(sb + j * kTileK * 2, mx, kt * kTileK, it.xrow + c0 + j, full);
             if (++stage == C::kStages) stage = 0, phase ^= 1u;
@@ -204,13 +212,13 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, const TcArgs a) {
             }
             tc_fence_after();
             const uint32_t sa = smem_base + stage * C::kStageBytes;
-            const uint32_t sb = sa + (UP ? 2 : 1) * kABytes;
+            const uint32_t sb = sa + 2 * kABytes;
 #pragma unroll
             for (int k = 0; k < kTileK / 16; ++k) {
               const uint32_t acc = (kt > 0 || k > 0) ? 1u : 0u;
               const uint64_t bd = smem_desc(sb + k * 32);
               umma_bf16(d0, smem_desc(sa + k * 32), bd, idesc, acc);
-              if (UP) umma_bf16(d0 + kNMax, smem_desc(sa + kABytes + k * 32), bd, idesc, acc);
+              if (it.ntile == 2) umma_bf16(d0 + kNMax, smem_desc(sa + kABytes + k * 32), bd, idesc, acc);
             }
             umma_commit(bar_empty + 8 * stage);   // frees the stage once these MMAs have read it
             if (++stage == C::kStages) stage = 0, phase ^= 1u;
@@ -270,12 +278,17 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, const TcArgs a) {
                 my_w = __ldg(a.sel_w + (size_t)it.l * a.S * a.K + pair);
               }
             }
+            float g2[16];
+            if (it.ntile == 2) tmem_ld16(t0 + kNMax + n0, g2);   // second row range: columns col + 128
             tmem_ld_wait();
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
               const int dst = __shfl_sync(0xffffffffu, my_dst, j);
               const float w = __shfl_sync(0xffffffffu, my_w, j);
-              if (dst >= 0) atomicAdd(a.y + (size_t)dst * a.d + col, w * g[j]);
+              if (dst >= 0) {
+                atomicAdd(a.y + (size_t)dst * a.d + col, w * g[j]);
+                if (it.ntile == 2) atomicAdd(a.y + (size_t)dst * a.d + col + kTileM, w * g2[j]);
+              }
             }
           }
         }
@@ -329,7 +342,7 @@ cudaError_t launch(const TcMaps& maps, const FfnParams& p, uint32_t* err, cudaSt
   }
   TcArgs a;
   a.L = p.L, a.S = p.S, a.E = p.E, a.K = p.K, a.n_sh = p.n_sh, a.d = p.d, a.I = p.I;
-  a.n_items = p.L * items_per_layer(p.E, p.n_sh, p.S, (UP ? p.I : p.d) / kTileM);
+  a.n_items = p.L * items_per_layer(p.E, p.n_sh, p.S, UP ? p.I / kTileM : (p.d / kTileM + 1) / 2);
   a.offsets = p.offsets, a.perm = p.perm, a.sel_w = p.sel_w, a.H = (__nv_bfloat16*)p.H, a.y = p.y, a.err = err;
   const int grid = a.n_items < sms ? a.n_items : sms;
   ffn_tc_kernel<UP><<<grid, kThreads, Cfg<UP>::kSmemBytes, st>>>(maps, a);
