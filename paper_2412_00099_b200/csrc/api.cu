@@ -104,7 +104,9 @@ Layout layout_of(const mcce_config& c) {
   o.inv = take(L * S * K * 4);
   o.Xg = take((L * S * K + 256) * d * esz);  // slack rows: tensor-core tiles read past a group's end
   o.H = take((rows + 256) * I * esz);
-  o.O = take(rows * d * 4);
+  // per-pair expert outputs are only needed by the fp32-pipe path (the tensor path combines in its epilogue)
+  const bool tensor_ffn = c.ffn_impl != MCCE_FFN_SIMT && tc_applicable(c);
+  o.O = take(tensor_ffn ? 0 : rows * d * 4);
   o.st_hidden = take(L * S * d * esz);
   o.st_sel = take(L * S * K * 4);
   o.st_w = take(L * S * K * 4);
