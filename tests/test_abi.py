@@ -42,7 +42,7 @@ def test_host_side_validation(lib):
     lib.mcce_strerror.restype = C.c_char_p
     ok = Config(24, 60, 4, 2, 4, 2048, 1408, 30, 256, 0.5, 0, 1, 1, 1, 0, 0)
     n = lib.mcce_workspace_bytes(C.byref(ok))
-    assert 500e6 < n < 2e9                      # gathered activations + intermediates for 6144 pairs
+    assert 250e6 < n < 1e9                      # gathered activations + intermediates for 6144 pairs
     for field, bad in [("n_experts", 257), ("top_k", 17), ("top_j", 5), ("d_model", 2050), ("cache_capacity", 0),
                        ("lam", -0.1), ("weight_dtype", 0), ("delta_mode", 2), ("n_streams", 0)]:
         cfg = Config(24, 60, 4, 2, 4, 2048, 1408, 30, 256, 0.5, 0, 1, 1, 1, 0, 0)
