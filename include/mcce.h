@@ -162,6 +162,20 @@ int mcce_get_cache_state(mcce_ctx* ctx, int32_t* order, uint8_t* ever, float* de
  * pos, pairs of one expert contiguous and in increasing (s,slot) order.  Synchronises. */
 int mcce_get_grouping(mcce_ctx* ctx, int32_t* offsets, int32_t* perm);
 
+/* Belady's optimal eviction (Sec. 4.8 "Optimal Cache Eviction") replayed on a recorded selection trace: the
+ * lossless bound that LRU cannot beat and that the paper's lossy rerouting can.  For every (stream, layer)
+ * and every capacity the trace is replayed from an empty cache; on a miss the expert is inserted, and while
+ * the cache is over capacity the resident expert whose next use lies farthest ahead is evicted, never one
+ * the current token itself selects.  Context-free.
+ *   sel_trace  DEVICE int32 [n_tokens, L, S, K]: the sel_idx output of mcce_route_step (K distinct experts)
+ *   capacities DEVICE int32 [n_capacities], each >= K
+ *   next_use_scratch DEVICE int32 [n_tokens, L, S, K], overwritten
+ *   misses     DEVICE int64 [n_capacities, L, S] out
+ * Asynchronous on the stream.  Capacities below K are the caller's error (the result is then undefined). */
+int mcce_belady_replay(const int32_t* sel_trace, int32_t n_tokens, int32_t n_layers, int32_t n_streams,
+                       int32_t n_experts, int32_t top_k, const int32_t* capacities, int32_t n_capacities,
+                       int32_t* next_use_scratch, int64_t* misses, void* cuda_stream);
+
 /* Seeded synthetic inputs (counter-based: Philox4x32-10 keyed by (seed, 0), counter = (element
  * block, t, tensor_id), Box-Muller with fixed-order fp32 series); no counterpart in the paper, whose
  * inputs are text corpora.  out DEVICE, dtype MCCE_F32/MCCE_BF16; elements [start, start+count) of the

@@ -23,7 +23,7 @@ RERANK_CACHE_PRIOR, RERANK_MAX_RANK, RERANK_CUMSUM = 0, 1, 2
 EXPORTS = [
     "mcce_workspace_bytes", "mcce_create", "mcce_destroy", "mcce_set_router", "mcce_set_experts", "mcce_reset",
     "mcce_route_step", "mcce_moe_forward", "mcce_decode_step_host", "mcce_cache_stats", "mcce_get_cache_state",
-    "mcce_get_grouping", "mcce_lifetime_stats", "mcce_profile", "mcce_profile_read", "mcce_uses_tensor_path", "mcce_selftest_wait_timeout", "mcce_route_trace_static",
+    "mcce_get_grouping", "mcce_lifetime_stats", "mcce_belady_replay", "mcce_profile", "mcce_profile_read", "mcce_uses_tensor_path", "mcce_selftest_wait_timeout", "mcce_route_trace_static",
     "mcce_route_trace_static_limit", "mcce_gen_normal", "mcce_gen_hidden_step", "mcce_gen_philox_words", "mcce_strerror",
     "mcce_last_cuda_error",
 ]
@@ -74,6 +74,7 @@ def load():
         lib.mcce_get_cache_state.argtypes = [vp, vp, vp, vp, C.POINTER(C.c_int64)]
         lib.mcce_get_grouping.argtypes = [vp, vp, vp]
         lib.mcce_lifetime_stats.argtypes = [vp, vp, vp]
+        lib.mcce_belady_replay.argtypes = [vp, i32, i32, i32, i32, i32, vp, i32, vp, vp, vp]
         lib.mcce_uses_tensor_path.argtypes = [vp]
         lib.mcce_selftest_wait_timeout.argtypes = [vp, C.c_uint64]
         lib.mcce_route_trace_static_limit.restype = C.c_size_t
@@ -306,3 +307,18 @@ def route_trace_static(*, L, E, K, J, C_cap, S, lam, logits=None, hidden=None, W
                                               _ptr(fixed_delta), _ptr(sel), _ptr(w),
                                               C.byref(totals) if want_totals else None, _stream()))
     return (sel, w, totals.as_tuple()) if want_totals else (sel, w)
+
+
+def belady_replay(sel_trace: torch.Tensor, n_experts: int, capacities) -> torch.Tensor:
+    """Misses of Belady's optimal eviction on a selection trace [T,L,S,K] (int32, device), for each capacity:
+    int64 tensor [n_capacities, L, S]."""
+    assert sel_trace.dtype == torch.int32 and sel_trace.dim() == 4
+    T, L, S, K = sel_trace.shape
+    caps = torch.tensor(list(capacities), dtype=torch.int32, device=sel_trace.device)
+    assert int(caps.min()) >= K, "Belady with a cache smaller than the K experts of one token is undefined"
+    scratch = torch.empty_like(sel_trace)
+    out = torch.empty((len(caps), L, S), dtype=torch.int64, device=sel_trace.device)
+    with torch.cuda.device(sel_trace.device):
+        _check(load().mcce_belady_replay(_ptr(sel_trace.contiguous()), T, L, S, n_experts, K, _ptr(caps), len(caps),
+                                         _ptr(scratch), _ptr(out), _stream()))
+    return out

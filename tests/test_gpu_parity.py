@@ -330,6 +330,29 @@ def test_decode_step_from_host_buffers():
         assert torch.allclose(yh, y.cpu(), rtol=1e-5, atol=1e-6)
 
 
+@pytest.mark.parametrize("E,K,S,T", [(8, 2, 5, 60), (60, 4, 7, 80), (130, 7, 3, 50), (16, 1, 4, 100)])
+def test_belady_replay_matches_the_oracle(E, K, S, T):
+    """Optimal-eviction miss counts on the trace the route kernel produces at lambda = 0, for several cache
+    sizes at once, against the oracle's farthest-next-use replay (itself pinned by exhaustive search)."""
+    from oracle import oracle as orc
+    L = 2
+    wl = synth.TINY.with_(L=L, E=E, K=K, J=0, C=max(K, E // 2), S=S, lam=0.0, d=64, I=64)
+    eng = mb.engine_for(wl)
+    z = ar1_logits(E + K, T, L, S, E, rho=0.6)
+    sel, _ = eng.route_step(logits=H.to_dev(z), n_steps=T)
+    caps = sorted({K, K + 1, max(K, E // 4), max(K, E // 2), E})
+    got = mb.belady_replay(sel, E, caps).cpu().numpy()
+    tr = sel.cpu().numpy()
+    lru_total, _ = eng.cache_stats()
+    for ci, c in enumerate(caps):
+        for l in range(L):
+            for s in range(S):
+                assert got[ci, l, s] == orc.belady_misses(tr[:, l, s], E, c)
+    # lossless bound: at the engine's capacity Belady cannot do worse than the LRU run that made the trace
+    assert got[caps.index(wl.C)].sum() <= lru_total[2]
+    assert (np.diff(got.sum(axis=(1, 2))) <= 0).all()            # more cache, never more misses
+
+
 def test_bounded_wait_gives_up_and_the_context_survives():
     """A wait that can never be satisfied ends after its limit with an error status instead of hanging;
     afterwards the same context routes correctly."""
