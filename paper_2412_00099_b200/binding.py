@@ -248,6 +248,15 @@ class Engine:
         sd = max(0.0, s2 / n - mean * mean) ** 0.5 if n else 0.0
         return (n, mean, sd), per
 
+    def calibrated_delta(self) -> np.ndarray:
+        """Per-layer logit range from the running statistics gathered so far (mean over streams of the
+        cumulative mean of max(z) - min(z)): the constants for a context in DELTA_FIXED mode, i.e. the
+        "estimate over a calibration set" variant of the paper's appendix on logit-range estimation."""
+        _, _, dsum, cnt = self.cache_state()
+        if cnt == 0:
+            raise McceError("no tokens routed yet: nothing to calibrate from")
+        return (dsum.astype(np.float64).mean(axis=1) / cnt).astype(np.float32)
+
     def grouping(self):
         offsets = np.empty((self.L, self.E + 1), np.int32)
         perm = np.empty((self.L, self.S * self.K), np.int32)

@@ -139,6 +139,25 @@ def test_cumsum_threshold_reached_exactly_on_gpu():
         assert sel.flatten().tolist() == [want]
 
 
+def test_calibrated_delta_feeds_fixed_mode():
+    """Logit range estimated on a warm-up trace (running mode), then used as per-layer constants."""
+    wl = synth.QWEN.with_(L=3, S=16, d=128, lam=0.5)
+    Wr = wl.router()
+    xs = list(wl.hidden_trace(24))
+    warm, o_warm = mb.engine_for(wl, ffn_impl=mb.FFN_SIMT), H.oracle_for(wl)
+    warm.set_router(H.to_dev(Wr))
+    for x in xs[:12]:
+        sel, w, z = warm.route_step(hidden=H.to_dev(x)[None], want_logits=True)
+        o_warm.route(z[0].cpu().numpy())
+    delta = warm.calibrated_delta()
+    ref = (o_warm.sum_range.astype(np.float64).mean(axis=1) / o_warm.count[0, 0]).astype(np.float32)
+    assert np.array_equal(delta, ref) and (delta > 0).all()
+    eng = mb.engine_for(wl, ffn_impl=mb.FFN_SIMT, delta_mode=mb.DELTA_FIXED)
+    eng.set_router(H.to_dev(Wr), H.to_dev(delta))
+    o = H.oracle_for(wl, delta_mode=1, fixed_delta=delta)
+    H.check_route_follow(eng, o, Wr, iter(xs[12:]), wl.bf16)
+
+
 def test_route_initial_state_and_resume():
     wl = synth.TINY.with_(L=2, E=24, K=3, J=1, C=7, S=5, lam=0.5)
     rng = np.random.default_rng(0)
