@@ -12,7 +12,8 @@
  * sequential because the cache state carries over.
  *
  * Ownership: the caller owns every buffer, including the workspace, and keeps them alive until
- * mcce_destroy.  The library allocates no device memory and creates no streams.  Weights are borrowed.
+ * mcce_destroy.  The library allocates no device memory and creates no streams (except the two copy
+ * streams of mcce_pipeline_submit_host).  Weights are borrowed.
  * Errors: every call returns 0 on success or a negative MCCE_E* code; nothing throws, aborts or prints.
  * Kernel launches are asynchronous on the given stream unless a function says that it synchronises.
  * A context is not thread-safe; distinct contexts are independent.
@@ -138,6 +139,21 @@ int mcce_moe_forward(mcce_ctx* ctx, const void* hidden, const int32_t* sel_idx, 
  * workspace.  hidden_host / y_host should be pinned.  Synchronises the stream before returning. */
 int mcce_decode_step_host(mcce_ctx* ctx, const void* hidden_host, float* y_host, int32_t* sel_idx_host,
                           void* cuda_stream);
+
+/* The same decode step, pipelined over successive tokens: copies overlap the compute of neighbouring steps.
+ * mcce_pipeline_submit_host enqueues, without waiting, the upload of hidden_host [L,S,d] on an internal
+ * copy-in stream, route + experts on cuda_stream once the upload has landed, and the download of y
+ * [L,S,d] (and sel_idx [L,S,K] if non-NULL) on an internal copy-out stream once the step has finished.
+ * Two staging slots alternate: a call blocks only if the step submitted two calls earlier has not yet left
+ * the device, so the upload of token t+1 and the download of token t-1 run while token t computes.  The
+ * host buffers of a submitted step must stay valid, and y_host must not be read, until mcce_pipeline_wait
+ * (or the second following submit) returns.  hidden_host / y_host must be pinned for the copies to be
+ * asynchronous.  The two copy streams and their events are the only CUDA objects the library creates (on
+ * the first submit); it still allocates no device memory.  Always use the same cuda_stream per context. */
+int mcce_pipeline_submit_host(mcce_ctx* ctx, const void* hidden_host, float* y_host, int32_t* sel_idx_host,
+                              void* cuda_stream);
+/* Waits until every submitted step has been copied back. */
+int mcce_pipeline_wait(mcce_ctx* ctx);
 
 /* Eq. 4 counters, summed over streams: total and per layer (HOST [L], may be NULL).  Synchronises.
  * Also reports MCCE_ETIMEOUT if any kernel of this context gave up on a bounded wait. */

@@ -22,7 +22,7 @@ RERANK_CACHE_PRIOR, RERANK_MAX_RANK, RERANK_CUMSUM = 0, 1, 2
 
 EXPORTS = [
     "mcce_workspace_bytes", "mcce_create", "mcce_destroy", "mcce_set_router", "mcce_set_experts", "mcce_reset",
-    "mcce_route_step", "mcce_moe_forward", "mcce_decode_step_host", "mcce_cache_stats", "mcce_get_cache_state",
+    "mcce_route_step", "mcce_moe_forward", "mcce_decode_step_host", "mcce_pipeline_submit_host", "mcce_pipeline_wait", "mcce_cache_stats", "mcce_get_cache_state",
     "mcce_get_grouping", "mcce_lifetime_stats", "mcce_belady_replay", "mcce_profile", "mcce_profile_read", "mcce_uses_tensor_path", "mcce_selftest_wait_timeout", "mcce_route_trace_static",
     "mcce_route_trace_static_limit", "mcce_gen_normal", "mcce_gen_hidden_step", "mcce_gen_philox_words", "mcce_strerror",
     "mcce_last_cuda_error",
@@ -70,6 +70,8 @@ def load():
         lib.mcce_route_step.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp]
         lib.mcce_moe_forward.argtypes = [vp] * 6
         lib.mcce_decode_step_host.argtypes = [vp] * 5
+        lib.mcce_pipeline_submit_host.argtypes = [vp] * 5
+        lib.mcce_pipeline_wait.argtypes = [vp]
         lib.mcce_cache_stats.argtypes = [vp, C.POINTER(Stats), C.POINTER(Stats)]
         lib.mcce_get_cache_state.argtypes = [vp, vp, vp, vp, C.POINTER(C.c_int64)]
         lib.mcce_get_grouping.argtypes = [vp, vp, vp]
@@ -207,6 +209,16 @@ class Engine:
         assert not hidden_host.is_cuda and not y_host.is_cuda
         _check(self.lib.mcce_decode_step_host(self.ctx, _ptr(hidden_host), _ptr(y_host), _ptr(sel_host), _stream()),
                self.ctx)
+
+    def pipeline_submit_host(self, hidden_host, y_host, sel_host=None):
+        """Asynchronous variant of decode_step_host: copies overlap the compute of neighbouring steps; call
+        pipeline_wait() before reading y_host."""
+        assert not hidden_host.is_cuda and not y_host.is_cuda
+        _check(self.lib.mcce_pipeline_submit_host(self.ctx, _ptr(hidden_host), _ptr(y_host), _ptr(sel_host),
+                                                  _stream()), self.ctx)
+
+    def pipeline_wait(self):
+        _check(self.lib.mcce_pipeline_wait(self.ctx), self.ctx)
 
     # -- state ------------------------------------------------------------------------------------------
     def cache_stats(self):

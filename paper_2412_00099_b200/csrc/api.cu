@@ -28,6 +28,13 @@ struct mcce_ctx {
   void* stage_hidden;
   int32_t* stage_sel;
   float *stage_w, *stage_y;
+  // second staging slot and the host-side machinery of the pipelined host entry point
+  void* stage_hidden2;
+  int32_t* stage_sel2;
+  float *stage_w2, *stage_y2;
+  cudaStream_t pipe_in, pipe_out;   // copy streams, created on first use
+  cudaEvent_t pipe_h2d[2], pipe_done[2], pipe_compute[2];
+  int pipe_ready, pipe_slot, pipe_busy[2];
   // borrowed weights
   const float *Wr, *fixed_delta;
   const void *Wg, *Wu, *Wd, *shWg, *shWu, *shWd;
@@ -77,7 +84,7 @@ bool valid(const mcce_config* c) {
 }
 
 struct Layout {
-  size_t stamp, ever, sum_range, miss, cold, err, stats, offsets, perm, inv, Xg, H, O, st_hidden, st_sel, st_w, st_y,
+  size_t stamp, ever, sum_range, miss, cold, err, stats, offsets, perm, inv, Xg, H, O, st_hidden, st_sel, st_w, st_y, st_hidden2, st_sel2, st_w2, st_y2,
       wr_terms, z_buf, load_tok, life, total;
 };
 
@@ -111,6 +118,10 @@ Layout layout_of(const mcce_config& c) {
   o.st_sel = take(L * S * K * 4);
   o.st_w = take(L * S * K * 4);
   o.st_y = take(L * S * d * 4);
+  o.st_hidden2 = take(L * S * d * esz);
+  o.st_sel2 = take(L * S * K * 4);
+  o.st_w2 = take(L * S * K * 4);
+  o.st_y2 = take(L * S * d * 4);
   const bool rg = router_gemm_applicable(c);
   o.wr_terms = take(rg ? 3 * L * E * d * 2 : 0);
   o.z_buf = take(rg ? (size_t)router_gemm_steps_max() * L * S * E * 4 : 0);
@@ -205,6 +216,8 @@ extern "C" int mcce_create(const mcce_config* cfg, void* workspace, size_t works
   ctx->Xg = w + lo.Xg, ctx->H = w + lo.H, ctx->O = (float*)(w + lo.O);
   ctx->stage_hidden = w + lo.st_hidden, ctx->stage_sel = (int32_t*)(w + lo.st_sel);
   ctx->stage_w = (float*)(w + lo.st_w), ctx->stage_y = (float*)(w + lo.st_y);
+  ctx->stage_hidden2 = w + lo.st_hidden2, ctx->stage_sel2 = (int32_t*)(w + lo.st_sel2);
+  ctx->stage_w2 = (float*)(w + lo.st_w2), ctx->stage_y2 = (float*)(w + lo.st_y2);
   ctx->use_tc = cfg->ffn_impl != MCCE_FFN_SIMT && tc_applicable(*cfg);
   ctx->use_tc_router = router_gemm_applicable(*cfg);
   ctx->wr_terms = w + lo.wr_terms, ctx->z_buf = (float*)(w + lo.z_buf);
@@ -225,6 +238,16 @@ extern "C" int mcce_create(const mcce_config* cfg, void* workspace, size_t works
 
 extern "C" int mcce_destroy(mcce_ctx* ctx) {
   if (!ctx) return MCCE_EINVAL;
+  if (ctx->pipe_ready) {
+    mcce_pipeline_wait(ctx);
+    cudaStreamDestroy(ctx->pipe_in);
+    cudaStreamDestroy(ctx->pipe_out);
+    for (int i = 0; i < 2; ++i) {
+      cudaEventDestroy(ctx->pipe_h2d[i]);
+      cudaEventDestroy(ctx->pipe_done[i]);
+      cudaEventDestroy(ctx->pipe_compute[i]);
+    }
+  }
   if (ctx->profiling)
     for (int i = 0; i < kMaxPairs; ++i) {
       cudaEventDestroy(ctx->ev[i][0]);
@@ -395,6 +418,67 @@ extern "C" int mcce_decode_step_host(mcce_ctx* ctx, const void* hidden_host, flo
   if (sel_idx_host)
     CK(cudaMemcpyAsync(sel_idx_host, ctx->stage_sel, LS * c.top_k * 4, cudaMemcpyDeviceToHost, st));
   CK(cudaStreamSynchronize(st));
+  return MCCE_OK;
+}
+
+// ---- pipelined host entry point: two staging slots, a copy-in and a copy-out stream ---------------------
+static int pipe_setup(mcce_ctx* ctx) {
+  if (ctx->pipe_ready) return MCCE_OK;
+  CK(cudaSetDevice(ctx->cfg.device));
+  CK(cudaStreamCreateWithFlags(&ctx->pipe_in, cudaStreamNonBlocking));
+  CK(cudaStreamCreateWithFlags(&ctx->pipe_out, cudaStreamNonBlocking));
+  for (int i = 0; i < 2; ++i) {
+    CK(cudaEventCreateWithFlags(&ctx->pipe_h2d[i], cudaEventDisableTiming));
+    CK(cudaEventCreateWithFlags(&ctx->pipe_done[i], cudaEventDisableTiming));
+    CK(cudaEventCreateWithFlags(&ctx->pipe_compute[i], cudaEventDisableTiming));
+  }
+  ctx->pipe_ready = 1;
+  return MCCE_OK;
+}
+
+extern "C" int mcce_pipeline_wait(mcce_ctx* ctx) {
+  if (!ctx) return MCCE_EINVAL;
+  if (!ctx->pipe_ready) return MCCE_OK;
+  for (int i = 0; i < 2; ++i)
+    if (ctx->pipe_busy[i]) {
+      CK(cudaEventSynchronize(ctx->pipe_done[i]));
+      ctx->pipe_busy[i] = 0;
+    }
+  return MCCE_OK;
+}
+
+extern "C" int mcce_pipeline_submit_host(mcce_ctx* ctx, const void* hidden_host, float* y_host, int32_t* sel_idx_host,
+                                         void* cuda_stream) {
+  if (!ctx || !hidden_host || !y_host) return MCCE_EINVAL;
+  int rc = pipe_setup(ctx);
+  if (rc != MCCE_OK) return rc;
+  const mcce_config& c = ctx->cfg;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  const size_t LS = (size_t)c.n_layers * c.n_streams, esz = c.hidden_dtype == MCCE_BF16 ? 2 : 4;
+  const int i = ctx->pipe_slot;
+  void* sh = i ? ctx->stage_hidden2 : ctx->stage_hidden;
+  int32_t* ss = i ? ctx->stage_sel2 : ctx->stage_sel;
+  float* sw = i ? ctx->stage_w2 : ctx->stage_w;
+  float* sy = i ? ctx->stage_y2 : ctx->stage_y;
+  // the slot's previous step (two submits ago) must have left the device before its buffers are reused
+  if (ctx->pipe_busy[i]) {
+    CK(cudaEventSynchronize(ctx->pipe_done[i]));
+    ctx->pipe_busy[i] = 0;
+  }
+  CK(cudaMemcpyAsync(sh, hidden_host, LS * c.d_model * esz, cudaMemcpyHostToDevice, ctx->pipe_in));
+  CK(cudaEventRecord(ctx->pipe_h2d[i], ctx->pipe_in));
+  CK(cudaStreamWaitEvent(st, ctx->pipe_h2d[i], 0));
+  rc = mcce_route_step(ctx, 1, sh, nullptr, ss, sw, nullptr, cuda_stream);
+  if (rc != MCCE_OK) return rc;
+  rc = mcce_moe_forward(ctx, sh, ss, sw, sy, cuda_stream);
+  if (rc != MCCE_OK) return rc;
+  CK(cudaEventRecord(ctx->pipe_compute[i], st));
+  CK(cudaStreamWaitEvent(ctx->pipe_out, ctx->pipe_compute[i], 0));
+  CK(cudaMemcpyAsync(y_host, sy, LS * c.d_model * 4, cudaMemcpyDeviceToHost, ctx->pipe_out));
+  if (sel_idx_host) CK(cudaMemcpyAsync(sel_idx_host, ss, LS * c.top_k * 4, cudaMemcpyDeviceToHost, ctx->pipe_out));
+  CK(cudaEventRecord(ctx->pipe_done[i], ctx->pipe_out));
+  ctx->pipe_busy[i] = 1;
+  ctx->pipe_slot = i ^ 1;
   return MCCE_OK;
 }
 

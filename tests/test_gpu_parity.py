@@ -385,6 +385,27 @@ def test_bounded_wait_gives_up_and_the_context_survives():
     H.check_route_exact(eng, H.oracle_for(wl), z)
 
 
+def test_pipelined_host_steps_match_synchronous_ones():
+    wl = synth.QWEN.with_(L=2, S=16, E=12, K=4, C=6, d=256, I=256, n_shared=1)
+    Wr, W = wl.router(), H.weights_for(wl)
+    a, b = mb.engine_for(wl), mb.engine_for(wl)
+    for e in (a, b):
+        e.set_router(H.to_dev(Wr))
+        e.set_experts(**{k: (None if v is None else H.to_dev(v)) for k, v in W.items()})
+    T = 7
+    xs = torch.stack([torch.from_numpy(x.view(np.int16)).view(torch.bfloat16) for x in wl.hidden_trace(T)]).pin_memory()
+    y_sync = torch.empty((T, wl.L, wl.S, wl.d), dtype=torch.float32).pin_memory()
+    s_sync = torch.empty((T, wl.L, wl.S, wl.K), dtype=torch.int32).pin_memory()
+    y_pipe, s_pipe = torch.zeros_like(y_sync).pin_memory(), torch.zeros_like(s_sync).pin_memory()
+    for t in range(T):
+        a.decode_step_host(xs[t], y_sync[t], s_sync[t])
+        b.pipeline_submit_host(xs[t], y_pipe[t], s_pipe[t])
+    b.pipeline_wait()
+    assert torch.equal(s_sync, s_pipe)
+    assert torch.allclose(y_sync, y_pipe, rtol=1e-5, atol=1e-6)
+    assert a.cache_stats()[0] == b.cache_stats()[0]
+
+
 # ---- argument checking: errors come back as codes, nothing is launched ------------------------------------
 def test_bad_arguments_are_rejected():
     with pytest.raises(mb.McceError):
