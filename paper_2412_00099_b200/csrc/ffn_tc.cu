@@ -328,18 +328,10 @@ bool make_map(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, ui
 
 template <bool UP>
 cudaError_t launch(const TcMaps& maps, const FfnParams& p, uint32_t* err, cudaStream_t st) {
-  static int sms = 0;
-  if (!sms) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    cudaError_t e = cudaFuncSetAttribute(ffn_tc_kernel<UP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)Cfg<UP>::kSmemBytes);
-    if (e != cudaSuccess) {
-      sms = 0;
-      return e;
-    }
-  }
+  static int cache[64] = {0};   // one per instantiation of this launcher, i.e. per kernel
+  int sms = 0;
+  cudaError_t e0 = sm_count_and_smem_optin(ffn_tc_kernel<UP>, Cfg<UP>::kSmemBytes, cache, &sms);
+  if (e0 != cudaSuccess) return e0;
   TcArgs a;
   a.L = p.L, a.S = p.S, a.E = p.E, a.K = p.K, a.n_sh = p.n_sh, a.d = p.d, a.I = p.I;
   a.n_items = p.L * items_per_layer(p.E, p.n_sh, p.S, UP ? p.I / kTileM : (p.d / kTileM + 1) / 2);

@@ -305,18 +305,10 @@ int router_gemm_plan(const mcce_config& c, const float* Wr, void* terms, RouterG
 
 cudaError_t router_gemm_launch(RouterGemmPlan& plan, const mcce_config& c, const void* hidden, int n_steps, float* Z,
                                int* k_split, uint32_t* err, cudaStream_t st) {
-  static int sms = 0;
-  if (!sms) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    cudaError_t e = cudaFuncSetAttribute(router_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)kSmemBytes);
-    if (e != cudaSuccess) {
-      sms = 0;
-      return e;
-    }
-  }
+  static int cache[64] = {0};
+  int sms = 0;
+  cudaError_t e0 = sm_count_and_smem_optin(router_gemm_kernel, kSmemBytes, cache, &sms);
+  if (e0 != cudaSuccess) return e0;
   const uint64_t rows = (uint64_t)n_steps * c.n_layers * c.n_streams;
   if (plan.hidden_ptr != hidden || plan.hidden_rows != rows) {
     EncodeFn fn = encode_fn();

@@ -130,5 +130,27 @@ inline EncodeFn encode_fn() {
   return fn;
 }
 
+
+// Number of SMs of the current device; the first call on a device also opts `kernel` in to `smem` bytes of
+// dynamic shared memory (an attribute that is set per device and per kernel: `sms` is the caller's
+// zero-initialised per-kernel cache).
+template <typename Kernel>
+inline cudaError_t sm_count_and_smem_optin(Kernel kernel, size_t smem, int (&sms)[64], int* sms_out) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  if (!sms[dev]) {
+    int n = 0;
+    e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    sms[dev] = n;
+  }
+  *sms_out = sms[dev];
+  return cudaSuccess;
+}
+
 }  // namespace tc
 }  // namespace mcce

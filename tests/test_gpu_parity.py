@@ -227,6 +227,25 @@ def test_model_shaped_routing_from_hidden_states(base, kw):
     print("%s: %d steps, %d near ties, max logit err %.2e" % (wl.name, steps, near, dz))
 
 
+def test_many_tokens_per_launch_from_hidden_states():
+    """n_steps beyond one logits-buffer chunk in a single call against one call per token: the cache
+    recurrence must be the same however the tokens are batched into launches."""
+    wl = synth.QWEN.with_(L=2, S=40, d=512)
+    Wr = H.to_dev(wl.router())
+    xs = np.stack(list(wl.hidden_trace(21)))
+    x = torch.from_numpy(xs.view(np.int16)).cuda().view(torch.bfloat16)
+    a, b = mb.engine_for(wl, ffn_impl=mb.FFN_SIMT), mb.engine_for(wl, ffn_impl=mb.FFN_SIMT)
+    a.set_router(Wr)
+    b.set_router(Wr)
+    sa, wa, za = a.route_step(hidden=x, n_steps=21, want_logits=True)
+    outs = [b.route_step(hidden=x[t:t + 1], want_logits=True) for t in range(21)]
+    zb = torch.cat([o[2] for o in outs])
+    assert torch.allclose(za, zb, rtol=0, atol=2e-6)       # the reduction may be split differently
+    assert torch.equal(sa, torch.cat([o[0] for o in outs]))
+    assert a.cache_stats()[0] == b.cache_stats()[0]
+    assert np.array_equal(a.cache_state()[0], b.cache_state()[0])
+
+
 # ---- grouping -------------------------------------------------------------------------------------------
 @pytest.mark.parametrize("L,S,E,K", [(1, 4, 8, 2), (3, 256, 60, 4), (2, 512, 64, 8), (2, 37, 200, 5), (1, 1, 1, 1)])
 def test_grouping_is_the_stable_counting_sort(L, S, E, K):
