@@ -1,5 +1,6 @@
-"""Parity at full size, in the configuration the benchmark times: the Qwen1.5-MoE-A2.7B-shaped workload
-(24 layers x 256 streams, 60+4 experts, bf16, tensor-core FFN path, one route + forward per token).
+"""Parity at full size, in the configuration the benchmark times (bf16, tensor-core paths, one route + forward
+per token): the Qwen1.5-MoE-A2.7B-shaped workload (24 layers x 256 streams, 60+4 experts) that the bench line is
+quoted on, and the OLMoE-, DeepSeek-V2-Lite- and Mixtral-8x7B-shaped ones.
 
 The library's inputs are generated on the device; the oracle's inputs for the sampled (layer, stream)
 pairs are regenerated on the host from the same seeded definition (the two generators agree bit for bit,
@@ -13,21 +14,28 @@ from paper_2412_00099_b200 import synth
 
 pytestmark = pytest.mark.gpu
 
-T_STEPS = 5
-SAMPLES = [(0, 0), (3, 17), (11, 128), (23, 255), (7, 64), (16, 201)]   # (layer, stream)
-FFN_SAMPLES = 4                                                        # pairs whose FFN output is recomputed
+def sample_pairs(wl):
+    """Six (layer, stream) pairs spread over the workload, corners included."""
+    L, S = wl.L, wl.S
+    return [(0, 0), (L // 8, S // 15), (L // 2, S // 2), (L - 1, S - 1), (L // 3, S // 4), (2 * L // 3, 4 * S // 5)]
+
+
+# workload, tokens, pairs whose FFN output is recomputed on the host (their expert matrices are regenerated there)
+CASES = [(synth.QWEN, 5, 4), (synth.OLMOE, 3, 2), (synth.DEEPSEEK, 3, 2), (synth.MIXTRAL, 3, 1)]
 
 
 def bits(t: torch.Tensor) -> np.ndarray:
     return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
 
 
-@pytest.mark.parametrize("wl", [synth.QWEN])
-def test_full_size_sampled_parity(wl):
+@pytest.mark.parametrize("wl,T_STEPS,FFN_SAMPLES", CASES, ids=[c[0].name for c in CASES])
+def test_full_size_sampled_parity(wl, T_STEPS, FFN_SAMPLES):
     from oracle import oracle as orc
     from paper_2412_00099_b200 import binding as mb
     import helpers as H
 
+    SAMPLES = sample_pairs(wl)
+    torch.cuda.empty_cache()            # the previous case's weights (tens of GB) must be gone first
     dev = torch.device("cuda")
     bf = torch.bfloat16
     eng = mb.engine_for(wl)
@@ -38,8 +46,8 @@ def test_full_size_sampled_parity(wl):
     sup, sdn = (wl.L, wl.n_shared, wl.I, wl.d), (wl.L, wl.n_shared, wl.d, wl.I)
     W = {"Wg": (synth.T_WG, up), "Wu": (synth.T_WU, up), "Wd": (synth.T_WD, dn), "shWg": (synth.T_SH_WG, sup),
          "shWu": (synth.T_SH_WU, sup), "shWd": (synth.T_SH_WD, sdn)}
-    Wt = {k: mb.gen_normal(torch.empty(shp, dtype=bf, device=dev), wl.seed, tid, std=wl.weight_std)
-          for k, (tid, shp) in W.items()}
+    Wt = {k: (mb.gen_normal(torch.empty(shp, dtype=bf, device=dev), wl.seed, tid, std=wl.weight_std)
+              if (wl.n_shared or not k.startswith("sh")) else None) for k, (tid, shp) in W.items()}
     eng.set_router(Wr)
     eng.set_experts(**Wt)
     assert np.array_equal(Wr.cpu().numpy(), wl.router())          # router: device generator == host generator
@@ -67,7 +75,7 @@ def test_full_size_sampled_parity(wl):
         topj = np.argsort(-z_h, -1, kind="stable")[..., :wl.J]
         assert all((topj[..., j:j + 1] == sel_h).any(-1).all() for j in range(wl.J))     # top-J always selected
         offsets, perm = eng.grouping()
-        for l in range(0, wl.L, 5):
+        for l in range(0, wl.L, 7):
             flat = sel_h[l].reshape(-1)
             assert np.array_equal(offsets[l], np.concatenate([[0], np.cumsum(np.bincount(flat, minlength=wl.E))]))
             assert np.array_equal(perm[l], np.argsort(flat, kind="stable"))
