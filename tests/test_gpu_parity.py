@@ -347,6 +347,24 @@ def test_tensor_core_path_agrees_with_simt_path(skew):
     H.ffn_close(ys[1], ys[0])
 
 
+@pytest.mark.parametrize("seed", range(10))
+def test_random_configurations_end_to_end(seed):
+    """Seeded random shapes and routing parameters (C < K, C >= E, J = 0, J = K, E not a multiple of 32, with
+    and without shared experts, ragged stream counts) through route + forward on the tensor-core paths."""
+    rng = np.random.default_rng(1000 + seed)
+    E = int(rng.integers(2, 97))
+    K = int(rng.integers(1, min(E, 8) + 1))
+    J = int(rng.integers(0, K + 1))
+    C = int(rng.choice([1, max(1, K - 1), K, max(K, E // 2), E, E + 3]))
+    wl = synth.QWEN.with_(L=int(rng.integers(1, 4)), S=int(rng.integers(1, 150)), E=E, K=K, J=J, C=C,
+                          d=128 * int(rng.integers(1, 5)), I=128 * int(rng.integers(1, 6)),
+                          n_shared=int(rng.integers(0, 3)), lam=float(rng.choice([0.0, 0.3, 0.5, 1.0, 2.0])),
+                          seed=100 + seed)
+    worst = run_forward_case(wl, 2, mb.FFN_TENSOR)
+    print("random config %d: L=%d S=%d E=%d K=%d J=%d C=%d d=%d I=%d sh=%d lam=%.1f -> max abs err %.2e" % (
+        seed, wl.L, wl.S, E, K, J, C, wl.d, wl.I, wl.n_shared, wl.lam, worst[0]))
+
+
 def test_decode_step_from_host_buffers():
     wl = synth.QWEN.with_(L=2, S=16, E=12, K=4, C=6, d=256, I=256, n_shared=1)
     Wr, W = wl.router(), H.weights_for(wl)
