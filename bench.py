@@ -326,6 +326,24 @@ def main_arm(args):
             # a memset of y, not a kernel, and is not counted)
             "gpu_launches": K * 6, "clocks": clocks}
 
+    # ---- routing alone, several tokens per launch (state stays in registers, the GEMM sees more tiles) -----
+    if not args.no_kernel_timing and wl.bf16 and n_tok >= 8:
+        eng.profile(True)
+        eng.profile_read(reset=True)
+        sel8 = torch.empty((8, wl.L, wl.S, wl.K), dtype=torch.int32, device=dev)
+        sw8 = torch.empty((8, wl.L, wl.S, wl.K), dtype=torch.float32, device=dev)
+        for it in range(13):
+            if it == 3:
+                eng.profile_read(reset=True)
+            eng.route_step(hidden=hidden[:8], n_steps=8, out=(sel8, sw8))
+        pr = eng.profile_read(reset=True)
+        eng.profile(False)
+        us = 1e3 * (pr["route"][0] / pr["route"][1] + pr["route_gemm"][0] / pr["route_gemm"][1])
+        state_bytes = 2 * (wl.E * 4 + EW * 4 + 12)
+        b8 = 8 * (wl.L * wl.S * (wl.d * esz + wl.K * 8) + wl.L * wl.E * wl.d * 4) + wl.L * wl.S * state_bytes
+        line["kernels"]["route"]["batched_8_tokens"] = {"us_per_launch": us, "achieved_gbs": b8 / (us * 1e-6) / 1e9,
+                                                        "algorithmic_bytes": b8}
+
     if args.lifetimes:
         (n_ev, mean, sd), _ = eng.lifetimes()
         line["cache_lifetime"] = {"evictions": n_ev, "mean_tokens": mean, "sd_tokens": sd,
