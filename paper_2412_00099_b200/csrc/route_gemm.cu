@@ -12,9 +12,9 @@
 // every kPhaseSlabs K-slabs: the epilogue warps add each phase's two partial sums into fp32 registers
 // with round-to-nearest adds while the MMA warp continues in the other TMEM buffer.
 //
-// Speed: an MMA that accumulates into the accumulator of the previous MMA waits for it (~100 cycles at
-// these small N), so consecutive k-steps alternate between kAccSets independent accumulator sets and
-// the 12 MMAs of a K-slab form chains of at most four.
+// Speed: a tcgen05.mma costs about 110 cycles to issue whatever N <= 128 is, so the kernel is bound by the
+// number of MMAs: the stream tile is as wide as TMEM allows with two accumulator buffers (N = 128), and the
+// reduction is split over up to eight CTAs per tile so that all SMs have work at one token per launch.
 //
 // Layout of the work: swapped GEMM as in the expert kernels -- router rows (experts) are MMA M (tiles of
 // 128, rows past E zero-filled by TMA at no memory cost), a block of streams is MMA N, the hidden
@@ -30,14 +30,14 @@ using namespace tc;
 
 namespace {
 
-constexpr int kTileM = 128, kTileK = 64, kNSMax = 64, kXBox = 16, kThreads = 192, kMaxStages = 12;
+constexpr int kTileM = 128, kTileK = 64, kNSMax = 128, kXBox = 16, kThreads = 192, kMaxStages = 12;
 constexpr uint32_t kRowBytes = kTileK * 2;                 // one 128-byte swizzle row
 // The stage ring.  A stage holds the three bf16 terms of a router slab -- only the RA rows that exist
 // (E rounded up to 8, at most 128) -- and the stream rows.  The MMA always reads 128 rows from a term's
 // start; rows past RA are whatever follows in the ring (finite or not, they only reach accumulator
 // rows of experts that do not exist), so the last 16 KB of the ring are never used as a stage start.
 constexpr uint32_t kRingBytes = 208 * 1024, kTermReadBytes = kTileM * kRowBytes;
-constexpr int kAccSets = 2;                                // independent accumulator sets (alternate k-steps)
+constexpr int kAccSets = 1;                                // independent accumulator sets (alternate k-steps)
 constexpr int kAccCols = 2 * kAccSets * kNSMax, kTmemCols = 2 * kAccCols;  // per buffer: sets x {hi, mid/lo}; 2 buffers
 constexpr int kPhaseSlabs = 4;                             // K-slabs (of 64) per accumulation phase
 constexpr size_t kSmemBytes = (size_t)kRingBytes + 1024 + 256;
@@ -202,15 +202,12 @@ router_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs a) {
 #pragma unroll
         for (int n0 = 0; n0 < kNSMax; n0 += 16) {
           if (n0 < a.NS) {
-            float hi[16], lo[16], hi1[16], lo1[16];
+            float hi[16], lo[16];
             tmem_ld16(t0 + n0, hi);
             tmem_ld16(t0 + kNSMax + n0, lo);
-            tmem_ld16(t0 + 2 * kNSMax + n0, hi1);
-            tmem_ld16(t0 + 3 * kNSMax + n0, lo1);
             tmem_ld_wait();
 #pragma unroll
-            for (int j = 0; j < 16; ++j)
-              zacc[n0 + j] = __fadd_rn(zacc[n0 + j], __fadd_rn(__fadd_rn(hi[j], hi1[j]), __fadd_rn(lo[j], lo1[j])));
+            for (int j = 0; j < 16; ++j) zacc[n0 + j] = __fadd_rn(zacc[n0 + j], __fadd_rn(hi[j], lo[j]));
           }
         }
         tc_fence_before();
@@ -325,21 +322,26 @@ cudaError_t router_gemm_launch(RouterGemmPlan& plan, const mcce_config& c, const
   }
   GemmArgs a;
   a.L = c.n_layers, a.S = c.n_streams, a.E = c.n_experts, a.d = c.d_model, a.n_steps = n_steps;
-  // streams per tile: as many as 64, fewer when that would leave most SMs without a tile
+  // streams per tile: as many as TMEM holds; narrower only when even the deepest K-split would leave most SMs idle
   int ns = c.n_streams >= kNSMax ? kNSMax : (c.n_streams + 15) & ~15;
   const int mt = (c.n_experts + kTileM - 1) / kTileM;
-  while (ns > 16 && n_steps * c.n_layers * mt * ((c.n_streams + ns - 1) / ns) < sms / 2) ns /= 2;
+  const int kt = c.d_model / kTileK;
+  int ks_max = 1;
+  while (ks_max < 8 && kt % (2 * ks_max) == 0 && kt / (2 * ks_max) >= 4 && n_steps * 2 * ks_max <= router_gemm_steps_max())
+    ks_max *= 2;
+  while (ns > 16 && n_steps * c.n_layers * mt * ((c.n_streams + ns - 1) / ns) * ks_max < sms / 2) ns /= 2;
   ns = (ns + 15) & ~15;
   a.NS = ns;
-  // split the reduction over up to four CTAs per tile while SMs would otherwise idle; the partial
+  // split the reduction over up to eight CTAs per tile while SMs would otherwise idle; the partial
   // logits are summed by the routing tail.  The logits buffer has router_gemm_steps_max() slots.
-  const int kt = c.d_model / kTileK;
   const int items = n_steps * c.n_layers * mt * ((c.n_streams + ns - 1) / ns);
+  // Cost of a split, from measurements on B200: a round of the persistent grid costs about 1 us per K-slab
+  // of its items (twelve MMAs) plus about 5 us of fill and drain, so one round of shorter items wins.
   int ks = 1;
-  double best = (double)((items + sms - 1) / sms);   // rounds of the persistent grid, in whole-tile units
-  for (int cand = 2; cand <= 4; cand *= 2) {
+  double best = (double)((items + sms - 1) / sms) * (kt * 1.0 + 5.0);
+  for (int cand = 2; cand <= 8; cand *= 2) {
     if (kt % cand || kt / cand < 4 || n_steps * cand > router_gemm_steps_max()) break;
-    const double cost = (double)((items * cand + sms - 1) / sms) / cand;
+    const double cost = (double)((items * cand + sms - 1) / sms) * (kt / cand * 1.0 + 5.0);
     if (cost < best - 1e-9) best = cost, ks = cand;
   }
   a.KS = ks, a.kt_per = kt / ks;
