@@ -15,8 +15,10 @@ namespace mcce {
 constexpr int kWarps = 8;
 constexpr int kDChunkMax = 4096;
 
-template <int NE>
-__global__ void __launch_bounds__(kWarps * 32) route_kernel(const RouteParams p, const int dchunk) {
+// HIDDEN: the kernel forms the logits itself (fp32-pipe front end); otherwise it only reads them, and is
+// compiled without that code so that it needs fewer registers and more warps fit on an SM.
+template <int NE, bool HIDDEN>
+__global__ void __launch_bounds__(kWarps * 32, HIDDEN ? 1 : 4) route_kernel(const RouteParams p, const int dchunk) {
   extern __shared__ __align__(16) float smem[];
   float* xs = smem;                          // [kWarps][dchunk]   hidden rows (fp32)
   float* zs = smem + (size_t)kWarps * dchunk;  // [kWarps][NE*32]   logits of this CTA's streams
@@ -58,7 +60,7 @@ __global__ void __launch_bounds__(kWarps * 32) route_kernel(const RouteParams p,
     const size_t row = ((size_t)t * p.L + l) * p.S + (active ? s : 0);
     float zr[NE];
 
-    if (p.hidden != nullptr) {
+    if (HIDDEN) {
       // ---- Eq. 3: logits of kWarps streams, router rows shared through the CTA ------------------
       for (int i = lane; i < NE * 32; i += 32) zs[warp * NE * 32 + i] = 0.f;
       const float* Wl = p.Wr + (size_t)l * E * p.d;
@@ -346,12 +348,17 @@ __global__ void __launch_bounds__(kWarps * 32) route_kernel(const RouteParams p,
 
 template <int NE>
 static cudaError_t launch_ne(const RouteParams& p, cudaStream_t st) {
+  if (!p.hidden) {
+    const int grid = p.L * ((p.S + kWarps - 1) / kWarps);
+    route_kernel<NE, false><<<grid, kWarps * 32, 0, st>>>(p, 0);
+    return cudaGetLastError();
+  }
   const int dchunk = p.hidden ? min((p.d + 3) & ~3, kDChunkMax) : 0;
   const size_t smem = p.hidden ? ((size_t)kWarps * dchunk + (size_t)kWarps * NE * 32) * sizeof(float) : 0;
-  cudaError_t e = cudaFuncSetAttribute(route_kernel<NE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t e = cudaFuncSetAttribute(route_kernel<NE, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   const int grid = p.L * ((p.S + kWarps - 1) / kWarps);
-  route_kernel<NE><<<grid, kWarps * 32, smem, st>>>(p, dchunk);
+  route_kernel<NE, true><<<grid, kWarps * 32, smem, st>>>(p, dchunk);
   return cudaGetLastError();
 }
 
