@@ -388,12 +388,10 @@ extern "C" int mcce_moe_forward(mcce_ctx* ctx, const void* hidden, const int32_t
   g.sel_idx = sel_idx, g.offsets = ctx->offsets, g.perm = ctx->perm, g.inv = ctx->inv;
   TIMED(MCCE_K_GROUP, st, launch_group(g, st));
   const FfnParams f = ffn_params(ctx, hidden, sel_w, y);
-  TIMED(MCCE_K_GATHER, st, launch_gather(f, st));
+  // on the tensor path the down kernel adds w * E_i(x) into y itself: the gather pass clears y on the way
+  TIMED(MCCE_K_GATHER, st, launch_gather(f, ctx->use_tc != 0, st));
   if (ctx->use_tc) {
-    // the down kernel adds w * E_i(x) into y itself: y starts at zero, no separate combine pass
     TIMED(MCCE_K_FFN_UP, st, tc_launch_up(ctx->tc, f, ctx->err, st));
-    TIMED(MCCE_K_COMBINE, st,
-          cudaMemsetAsync(y, 0, (size_t)c.n_layers * c.n_streams * c.d_model * sizeof(float), st));
     TIMED(MCCE_K_FFN_DOWN, st, tc_launch_down(ctx->tc, f, ctx->err, st));
   } else {
     TIMED(MCCE_K_FFN_UP, st, launch_ffn_simt_up(f, st));

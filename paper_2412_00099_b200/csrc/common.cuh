@@ -84,7 +84,7 @@ cudaError_t launch_wait_timeout_selftest(uint32_t* err, unsigned long long limit
                                          cudaStream_t st);
 cudaError_t launch_route(const RouteParams& p, cudaStream_t st);
 cudaError_t launch_group(const GroupParams& p, cudaStream_t st);
-cudaError_t launch_gather(const FfnParams& p, cudaStream_t st);
+cudaError_t launch_gather(const FfnParams& p, bool zero_y, cudaStream_t st);
 cudaError_t launch_ffn_simt_up(const FfnParams& p, cudaStream_t st);
 cudaError_t launch_ffn_simt_down(const FfnParams& p, cudaStream_t st);
 cudaError_t launch_combine(const FfnParams& p, cudaStream_t st);

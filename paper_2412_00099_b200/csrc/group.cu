@@ -74,8 +74,9 @@ cudaError_t launch_group(const GroupParams& p, cudaStream_t st) {
   return cudaGetLastError();
 }
 
-// Xg[l][pos][:] = hidden[l][perm[l][pos] / K][:]; one warp per row, 16-byte copies.
-__global__ void gather_kernel(const FfnParams p) {
+// Xg[l][pos][:] = hidden[l][perm[l][pos] / K][:]; one warp per row, 16-byte copies.  With zero_y the warp of
+// pair (s, k) also clears the k-th of K slices of y[l][s][:], for the expert kernel that accumulates into y.
+__global__ void gather_kernel(const FfnParams p, const int zero_y) {
   const int P = p.S * p.K;
   const size_t row = (size_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (row >= (size_t)p.L * P) return;
@@ -86,12 +87,18 @@ __global__ void gather_kernel(const FfnParams p) {
   const uint4* src = (const uint4*)((const char*)p.hidden + ((size_t)l * p.S + s) * bytes);
   uint4* dst = (uint4*)((char*)p.Xg + row * bytes);
   for (int i = lane; i < (int)(bytes / 16); i += 32) dst[i] = __ldg(src + i);
+  if (zero_y) {
+    const int k = p.perm[row] % p.K, n4 = p.d / 4;            // y row: d floats = n4 float4
+    const int lo = (int)((long long)n4 * k / p.K), hi = (int)((long long)n4 * (k + 1) / p.K);
+    float4* y = (float4*)(p.y + ((size_t)l * p.S + s) * p.d);
+    for (int i = lo + lane; i < hi; i += 32) y[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+  }
 }
 
-cudaError_t launch_gather(const FfnParams& p, cudaStream_t st) {
+cudaError_t launch_gather(const FfnParams& p, bool zero_y, cudaStream_t st) {
   const size_t rows = (size_t)p.L * p.S * p.K;
   const int wpb = 8;
-  gather_kernel<<<(unsigned)((rows + wpb - 1) / wpb), wpb * 32, 0, st>>>(p);
+  gather_kernel<<<(unsigned)((rows + wpb - 1) / wpb), wpb * 32, 0, st>>>(p, zero_y ? 1 : 0);
   return cudaGetLastError();
 }
 
