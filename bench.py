@@ -33,7 +33,7 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel (ffn_up), per layer,
 # from the ncu capture summarised in profiles/step_kernels_qwen_4layers.md (a 4-layer case; traffic
 # grows in proportion to the layer count).  Workloads without a capture of the current kernel: None.
-NCU_TRAFFIC_BYTES_PER_LAYER = {"qwen1.5-moe-a2.7b-shaped": (2976666000 + 23316736) / 4}
+NCU_TRAFFIC_BYTES_PER_LAYER = {"qwen1.5-moe-a2.7b-shaped": (2976824000 + 25219328) / 4}
 
 
 def parse_args():
