@@ -213,10 +213,10 @@ int mcce_gen_philox_words(uint32_t* out, uint64_t start_block, uint64_t n_blocks
 enum {
   MCCE_K_ROUTE = 0,    /* fused route kernel (with bf16 hidden states: its tail, on the logits of MCCE_K_ROUTE_GEMM) */
   MCCE_K_GROUP = 1,    /* histogram + scan + scatter                 */
-  MCCE_K_GATHER = 2,   /* activation rows into expert order          */
+  MCCE_K_GATHER = 2,   /* activation rows into expert order (clears y on the tensor-core path) */
   MCCE_K_FFN_UP = 3,   /* H = silu(X Wg^T) * (X Wu^T), all groups    */
   MCCE_K_FFN_DOWN = 4, /* O = H Wd^T, all groups                     */
-  MCCE_K_COMBINE = 5,  /* weighted sum over slots + shared experts   */
+  MCCE_K_COMBINE = 5,  /* weighted sum over slots + shared experts (fp32-pipe path; fused into FFN_DOWN otherwise) */
   MCCE_K_ROUTE_GEMM = 6, /* router logits on the tensor cores (bf16 hidden states) */
   MCCE_N_KERNELS = 7
 };
