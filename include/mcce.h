@@ -168,6 +168,13 @@ int mcce_cache_stats(mcce_ctx* ctx, mcce_stats* total /*HOST*/, mcce_stats* per_
 typedef struct { int64_t evictions, sum, sum_sq; } mcce_lifetime;
 int mcce_lifetime_stats(mcce_ctx* ctx, mcce_lifetime* total /*HOST*/, mcce_lifetime* per_layer /*HOST*/);
 
+/* Per-token miss trace (the data behind the paper's hit / miss timelines of Sec. 4.6): while a buffer is set,
+ * every routed token writes one word per (layer, stream) whose bit k says that the k-th selected expert was
+ * not in the cache.  trace: DEVICE uint32 [capacity_tokens, L, S], caller-owned; tokens beyond the capacity
+ * are not recorded; recording restarts at entry 0 when the buffer is set and after mcce_reset.  NULL with
+ * capacity 0 turns it off. */
+int mcce_set_miss_trace(mcce_ctx* ctx, uint32_t* trace, int64_t capacity_tokens);
+
 /* Canonical cache state: order HOST int32 [L,S,C] most-recently-used first, -1 padded; optional
  * ever HOST uint8 [L,S,E]; delta_sum HOST fp32 [L,S] and *delta_count (optional).  Synchronises. */
 int mcce_get_cache_state(mcce_ctx* ctx, int32_t* order, uint8_t* ever, float* delta_sum,

@@ -133,6 +133,7 @@ void orc_route_slab(const orc_config* c, const float* z_all /*[L,S,E]*/,
                     float* w_all /*[L,S,K]*/, float* margin_all /*[L,S] or NULL*/,
                     float* delta_all /*[L,S] or NULL*/, int64_t* load_tok_all /*[L,S,E] or NULL*/,
                     int64_t* life_all /*[L,S,3] or NULL: evictions, sum and sum of squares of lifetimes*/,
+                    uint32_t* miss_mask_all /*[L,S] or NULL: bit k set iff the k-th selected expert missed*/,
                     int s0, int s1) {
   const int L = c->n_layers, E = c->n_experts, K = c->top_k, J = c->top_j, S = c->n_streams;
   const int C = c->cache_capacity;
@@ -217,10 +218,13 @@ void orc_route_slab(const orc_config* c, const float* z_all /*[L,S,E]*/,
       /* Eq. 4 against the cache as it was before this token. */
       int64_t* cnt = counters_all + p * 4;
       int miss = 0, cold = 0;
+      uint32_t miss_mask = 0;
       for (int k = 0; k < K; ++k) {
         if (stamp[sel[k]] == 0) ++miss;
+        if (stamp[sel[k]] == 0) miss_mask |= 1u << k;
         if (!ever[sel[k]]) ++cold;
       }
+      if (miss_mask_all) miss_mask_all[p] = miss_mask;
       cnt[0] += 1;
       cnt[1] += K;
       cnt[2] += miss;

@@ -101,6 +101,7 @@ class Oracle:
         self.counters = np.zeros((L, S, 4), np.int64)
         self.load_tok = np.zeros((L, S, E), np.int64)
         self.life = np.zeros((L, S, 3), np.int64)
+        self.last_miss_mask = np.zeros((L, S), np.uint32)   # of the latest token: bit k = slot k missed
         self.fixed_delta = None if fixed_delta is None else np.ascontiguousarray(fixed_delta, np.float32)
         self.threads = threads
         self._pool = ThreadPoolExecutor(threads) if threads > 1 else None
@@ -166,7 +167,7 @@ class Oracle:
         self._par(lambda a, b: lib().orc_route_slab(
             C.byref(cc), _p(z), _p(self.fixed_delta), _p(self.stamp), _p(self.ever),
             _p(self.sum_range), _p(self.count), _p(self.tok), _p(self.counters), _p(sel), _p(w),
-            _p(margin), _p(delta), _p(self.load_tok), _p(self.life), a, b))
+            _p(margin), _p(delta), _p(self.load_tok), _p(self.life), _p(self.last_miss_mask), a, b))
         if want_margin:
             return sel, w, margin, delta
         return sel, w

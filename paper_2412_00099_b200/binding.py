@@ -23,7 +23,7 @@ RERANK_CACHE_PRIOR, RERANK_MAX_RANK, RERANK_CUMSUM = 0, 1, 2
 EXPORTS = [
     "mcce_workspace_bytes", "mcce_create", "mcce_destroy", "mcce_set_router", "mcce_set_experts", "mcce_reset",
     "mcce_route_step", "mcce_moe_forward", "mcce_decode_step_host", "mcce_pipeline_submit_host", "mcce_pipeline_wait", "mcce_cache_stats", "mcce_get_cache_state",
-    "mcce_get_grouping", "mcce_lifetime_stats", "mcce_belady_replay", "mcce_profile", "mcce_profile_read", "mcce_uses_tensor_path", "mcce_selftest_wait_timeout", "mcce_route_trace_static",
+    "mcce_get_grouping", "mcce_lifetime_stats", "mcce_set_miss_trace", "mcce_belady_replay", "mcce_profile", "mcce_profile_read", "mcce_uses_tensor_path", "mcce_selftest_wait_timeout", "mcce_route_trace_static",
     "mcce_route_trace_static_limit", "mcce_gen_normal", "mcce_gen_hidden_step", "mcce_gen_philox_words", "mcce_strerror",
     "mcce_last_cuda_error",
 ]
@@ -76,6 +76,7 @@ def load():
         lib.mcce_get_cache_state.argtypes = [vp, vp, vp, vp, C.POINTER(C.c_int64)]
         lib.mcce_get_grouping.argtypes = [vp, vp, vp]
         lib.mcce_lifetime_stats.argtypes = [vp, vp, vp]
+        lib.mcce_set_miss_trace.argtypes = [vp, vp, C.c_int64]
         lib.mcce_belady_replay.argtypes = [vp, i32, i32, i32, i32, i32, vp, i32, vp, vp, vp]
         lib.mcce_uses_tensor_path.argtypes = [vp]
         lib.mcce_selftest_wait_timeout.argtypes = [vp, C.c_uint64]
@@ -249,6 +250,13 @@ class Engine:
         n = np.zeros(len(self.KERNELS), np.int64)
         _check(self.lib.mcce_profile_read(self.ctx, _ptr(ms), _ptr(n), int(reset)), self.ctx)
         return {k: (float(ms[i]), int(n[i])) for i, k in enumerate(self.KERNELS)}
+
+    def record_misses(self, n_tokens: int) -> torch.Tensor:
+        """Allocates and registers a miss-trace buffer [n_tokens, L, S] (uint32 bit masks, viewed as int32):
+        bit k of entry (t, l, s) is set iff the k-th selected expert of that token missed the cache."""
+        self._trace = torch.zeros((n_tokens, self.L, self.S), dtype=torch.int32, device=self.device)
+        _check(self.lib.mcce_set_miss_trace(self.ctx, _ptr(self._trace), n_tokens), self.ctx)
+        return self._trace
 
     def lifetimes(self):
         """(evictions, mean, standard deviation) of cache lifetimes in tokens, and the raw per-layer sums."""

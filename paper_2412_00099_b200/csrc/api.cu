@@ -38,6 +38,9 @@ struct mcce_ctx {
   // borrowed weights
   const float *Wr, *fixed_delta;
   const void *Wg, *Wu, *Wd, *shWg, *shWu, *shWd;
+  // optional per-token miss trace (caller's buffer)
+  uint32_t* miss_trace;
+  int64_t trace_cap, trace_pos;
   // host-side counters
   uint64_t tok, delta_cnt, steps_since_reset;
   int last_cuda;
@@ -325,6 +328,7 @@ extern "C" int mcce_reset(mcce_ctx* ctx, const int32_t* init_order, int keep_del
   }
   ctx->tok = 0;
   ctx->steps_since_reset = 0;
+  ctx->trace_pos = 0;
   CK(cudaDeviceSynchronize());
   return MCCE_OK;
 }
@@ -348,6 +352,13 @@ extern "C" int mcce_route_step(mcce_ctx* ctx, int32_t n_steps, const void* hidde
   p.Wr = ctx->Wr, p.fixed_delta = ctx->fixed_delta;
   p.stamp = ctx->stamp, p.ever = ctx->ever, p.sum_range = ctx->sum_range, p.miss = ctx->miss, p.cold = ctx->cold;
   p.load_tok = ctx->load_tok, p.life = ctx->life;
+  const size_t LS_trace = (size_t)c.n_layers * c.n_streams;
+  auto trace_at = [&](int t0, int nt) {   // where tokens [t0, t0+nt) of this call go in the trace buffer
+    const int64_t pos = ctx->trace_pos + t0;
+    const bool on = ctx->miss_trace && pos < ctx->trace_cap;
+    p.miss_trace = on ? ctx->miss_trace + (size_t)pos * LS_trace : nullptr;
+    p.trace_avail = on ? (int)(ctx->trace_cap - pos < nt ? ctx->trace_cap - pos : nt) : 0;
+  };
   cudaStream_t st = (cudaStream_t)cuda_stream;
   if (hidden && ctx->use_tc_router && ctx->rg.ready) {
     // logits by the tensor-core GEMM, a few tokens at a time, then the fused tail on those logits
@@ -362,16 +373,19 @@ extern "C" int mcce_route_step(mcce_ctx* ctx, int32_t n_steps, const void* hidde
       p.sel_idx = sel_idx + (size_t)t0 * LS * c.top_k, p.sel_w = sel_w + (size_t)t0 * LS * c.top_k;
       p.logits_out = logits_out ? logits_out + (size_t)t0 * LS * c.n_experts : nullptr;
       p.tok0 = (uint32_t)(ctx->tok + t0), p.cnt0 = (uint32_t)(ctx->delta_cnt + t0);
+      trace_at(t0, nt);
       TIMED(MCCE_K_ROUTE, st, launch_route(p, st));
     }
   } else {
     p.n_steps = n_steps, p.hidden = hidden, p.logits_in = logits_in, p.n_partials = 1, p.partial_stride = 0;
     p.sel_idx = sel_idx, p.sel_w = sel_w, p.logits_out = logits_out;
     p.tok0 = (uint32_t)ctx->tok, p.cnt0 = (uint32_t)ctx->delta_cnt;
+    trace_at(0, n_steps);
     TIMED(MCCE_K_ROUTE, st, launch_route(p, st));
   }
   ctx->tok += n_steps;
   ctx->steps_since_reset += n_steps;
+  if (ctx->miss_trace) ctx->trace_pos += n_steps;
   if (c.delta_mode == MCCE_DELTA_RUNNING) ctx->delta_cnt += n_steps;
   return MCCE_OK;
 }
@@ -529,6 +543,14 @@ extern "C" int mcce_get_cache_state(mcce_ctx* ctx, int32_t* order, uint8_t* ever
   }
   if (delta_sum) CK(cudaMemcpy(delta_sum, ctx->sum_range, LS * 4, cudaMemcpyDeviceToHost));
   if (delta_count) *delta_count = (int64_t)ctx->delta_cnt;
+  return MCCE_OK;
+}
+
+extern "C" int mcce_set_miss_trace(mcce_ctx* ctx, uint32_t* trace, int64_t capacity_tokens) {
+  if (!ctx || capacity_tokens < 0 || (trace == nullptr) != (capacity_tokens == 0)) return MCCE_EINVAL;
+  ctx->miss_trace = trace;
+  ctx->trace_cap = capacity_tokens;
+  ctx->trace_pos = 0;
   return MCCE_OK;
 }
 

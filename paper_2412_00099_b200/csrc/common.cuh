@@ -35,6 +35,8 @@ struct RouteParams {
   uint32_t* cold;            // [L,S]
   uint32_t* load_tok;        // [L,S,E] token that loaded each resident expert, or null (lifetimes not tracked)
   unsigned long long* life;  // [L,S,3]  evictions, sum and sum of squares of cache lifetimes
+  uint32_t* miss_trace;      // [trace_avail,L,S] per-token miss bits of this launch's tokens, or null
+  int trace_avail;           // tokens of this launch that still fit the trace buffer
   int32_t* sel_idx;          // [n_steps,L,S,K]
   float* sel_w;              // [n_steps,L,S,K]
   float* logits_out;         // [n_steps,L,S,E] or null

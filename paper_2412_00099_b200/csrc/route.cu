@@ -260,7 +260,10 @@ __global__ void __launch_bounds__(kWarps * 32, HIDDEN ? 1 : 4) route_kernel(cons
       const uint32_t rb = __shfl_sync(kFull, resb, my_sel & 31);
       const uint32_t eb = __shfl_sync(kFull, everb, my_sel & 31);
       const bool sel_lane = lane < K;
-      miss_c += __popc(__ballot_sync(kFull, sel_lane && !((rb >> (my_sel >> 5)) & 1u)));
+      const uint32_t miss_bits = __ballot_sync(kFull, sel_lane && !((rb >> (my_sel >> 5)) & 1u));
+      miss_c += __popc(miss_bits);   // lane k holds the k-th selected expert: bit k = slot k missed
+      if (p.miss_trace != nullptr && t < p.trace_avail && lane == 0)
+        p.miss_trace[((size_t)t * p.L + l) * p.S + s] = miss_bits;
       cold_c += __popc(__ballot_sync(kFull, sel_lane && !((eb >> (my_sel >> 5)) & 1u)));
     }
 

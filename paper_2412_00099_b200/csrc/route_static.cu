@@ -74,7 +74,7 @@ extern "C" int mcce_route_trace_static(const mcce_config* cfg, int32_t n_steps, 
   p.L = cfg->n_layers, p.S = cfg->n_streams, p.E = cfg->n_experts, p.K = cfg->top_k, p.J = cfg->top_j;
   p.C = cfg->cache_capacity, p.d = cfg->d_model, p.n_steps = n_steps, p.lambda = cfg->lambda;
   p.delta_mode = cfg->delta_mode, p.renorm = cfg->renorm, p.hidden_bf16 = cfg->hidden_dtype == MCCE_BF16;
-  p.n_partials = 1, p.partial_stride = 0, p.load_tok = nullptr, p.life = nullptr;
+  p.n_partials = 1, p.partial_stride = 0, p.load_tok = nullptr, p.life = nullptr, p.miss_trace = nullptr, p.trace_avail = 0;
   p.rerank_mode = cfg->rerank_mode, p.max_rank = cfg->max_rank, p.cum_threshold = cfg->cum_threshold;
   p.hidden = hidden, p.logits_in = logits_in, p.Wr = Wr, p.fixed_delta = fixed_delta;
   p.stamp = (uint32_t*)(base + o_stamp), p.ever = (uint32_t*)(base + o_ever);

@@ -139,6 +139,33 @@ def test_cumsum_threshold_reached_exactly_on_gpu():
         assert sel.flatten().tolist() == [want]
 
 
+def test_miss_trace_matches_the_oracle():
+    """Per-token miss bits, through both routing front ends (given logits; hidden states via the GEMM)."""
+    wl = synth.QWEN.with_(L=2, S=19, d=128, C=9)
+    T = 20
+    eng, o = mb.engine_for(wl, ffn_impl=mb.FFN_SIMT), H.oracle_for(wl)
+    trace = eng.record_misses(T - 4)                         # shorter than the run: the tail is not recorded
+    z = ar1_logits(77, T, wl.L, wl.S, wl.E)
+    eng.route_step(logits=H.to_dev(z[:12]), n_steps=12)
+    for t in range(12, T):
+        eng.route_step(logits=H.to_dev(z[t:t + 1]))
+    want = np.zeros((T, wl.L, wl.S), np.uint32)
+    for t in range(T):
+        o.route(z[t])
+        want[t] = o.last_miss_mask
+    got = trace.cpu().numpy().view(np.uint32)
+    assert np.array_equal(got, want[:T - 4])
+    assert sum(bin(int(v)).count("1") for v in want.ravel()) == eng.cache_stats()[0][2]
+    # from hidden states (tensor-core logits): follow the library's logits, compare the bits
+    eng2, o2 = mb.engine_for(wl, ffn_impl=mb.FFN_SIMT), H.oracle_for(wl)
+    eng2.set_router(H.to_dev(wl.router()))
+    tr2 = eng2.record_misses(6)
+    for t, x in enumerate(wl.hidden_trace(6)):
+        _, _, zg = eng2.route_step(hidden=H.to_dev(x)[None], want_logits=True)
+        o2.route(zg[0].cpu().numpy())
+        assert np.array_equal(tr2[t].cpu().numpy().view(np.uint32), o2.last_miss_mask)
+
+
 def test_calibrated_delta_feeds_fixed_mode():
     """Logit range estimated on a warm-up trace (running mode), then used as per-layer constants."""
     wl = synth.QWEN.with_(L=3, S=16, d=128, lam=0.5)

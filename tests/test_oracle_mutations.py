@@ -22,6 +22,9 @@ MUTATIONS = [
      "w[k] = (float)(exp((double)zp[sel[k]] - (double)zmax)"),
     ("renormalisation denominators swapped", "(c->renorm ? denom_sel : denom_all)", "(c->renorm ? denom_all : denom_sel)"),
     ("hits counted as misses", "if (stamp[sel[k]] == 0) ++miss;", "if (stamp[sel[k]] != 0) ++miss;"),
+    ("miss trace marks the hits", "if (stamp[sel[k]] == 0) miss_mask |= 1u << k;", "if (stamp[sel[k]] != 0) miss_mask |= 1u << k;"),
+    ("miss trace indexed by expert instead of slot", "if (stamp[sel[k]] == 0) miss_mask |= 1u << k;",
+     "if (stamp[sel[k]] == 0) miss_mask |= 1u << (sel[k] & 31);"),
     ("in-token order reversed", "stamp[e] = (int64_t)E + tok * K + r + 1;", "stamp[e] = (int64_t)E + tok * K + (K - 1 - r) + 1;"),
     ("evicts the most recent expert", "if (victim < 0 || stamp[e] < stamp[victim]) victim = e;\n        }\n        if (resident <= C) break;\n        stamp[victim] = 0;\n        if (life_all)",
      "if (victim < 0 || stamp[e] > stamp[victim]) victim = e;\n        }\n        if (resident <= C) break;\n        stamp[victim] = 0;\n        if (life_all)"),
@@ -70,7 +73,8 @@ def run_pins():
              (pins.test_max_rank_mode_follows_algorithm_1, (4, 1)), (pins.test_cumsum_mode_follows_algorithm_2, (0.6,)),
              (pins.test_max_rank_over_all_ranks_is_the_saturated_cache_prior, (1,)),
              (pins.test_lifetimes_match_brute_force_over_resident_sets, ()),
-             (pins.test_cumsum_mode_reaches_the_threshold_exactly, ())]
+             (pins.test_cumsum_mode_reaches_the_threshold_exactly, ()),
+             (pins.test_miss_trace_matches_resident_sets, ())]
     failed = []
     for fn, args in calls:
         try:

@@ -616,3 +616,19 @@ def test_lifetimes_grow_with_lambda_on_tiny():
             o.route(o.logits(Wr, x))
         means.append(o.lifetimes()[1])
     assert means[1] > 1.5 * means[0]
+
+
+def test_miss_trace_matches_resident_sets():
+    """Per-token miss bits (slot k of the selection missed) against the resident set exported before the token."""
+    rng = np.random.default_rng(59)
+    E, K, C = 9, 3, 4
+    o = make(E=E, K=K, J=1, C=C, lam=0.4, L=1, S=2)
+    total = 0
+    for z in ar1_logits(rng, 80, 1, 2, E, rho=0.6):
+        before = [set(e for e in row.tolist() if e >= 0) for row in o.order()[0]]
+        sel, _ = o.route(z)
+        for s in range(2):
+            want = sum(1 << k for k in range(K) if int(sel[0, s, k]) not in before[s])
+            assert int(o.last_miss_mask[0, s]) == want
+            total += bin(want).count("1")
+    assert total == o.stats()[0][2]
