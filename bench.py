@@ -112,6 +112,16 @@ def oracle_sample(wl, steps: int, warmup: int, core_seconds: float = 20.0):
     dt = time.perf_counter() - t0
     desc = "layer 0, first %d of %d streams, %d tokens, routing + expert FFN, %d host threads" % (
         S_s, wl.S, steps, threads)
+    # the same code on one core (a fresh oracle on the first two streams, one token)
+    n1 = min(2, S_s)
+    o1 = orc.Oracle(orc.OracleConfig(1, wl.E, wl.K, wl.J, wl.n_shared, wl.d, wl.I, wl.C, n1, wl.lam, 0, 1,
+                                     1 if wl.bf16 else 0), threads=1)
+    x1 = np.ascontiguousarray(xs[-1][:, :n1])
+    t1 = time.perf_counter()
+    z1 = o1.logits(Wr, x1)
+    sel1, w1 = o1.route(z1)
+    o1.ffn(x1, sel1, w1, W["Wg"], W["Wu"], W["Wd"], sh["shWg"], sh["shWu"], sh["shWd"])
+    oracle_sample.single_core = n1 / (time.perf_counter() - t1)
     return S_s * steps / dt, threads, desc, dt / steps
 
 
@@ -128,7 +138,8 @@ def reference_arm(args):
             "warmup": warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": config_of(wl, {"sample": desc}),
-            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc,
+                             "value_one_core": oracle_sample.single_core},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line))
@@ -381,7 +392,8 @@ def main_arm(args):
     # ---- the oracle on the host cores, beside it ------------------------------------------------------------
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         v, threads, desc, _ = oracle_sample(wl, steps=4, warmup=1)
-        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc}
+        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc,
+                                "value_one_core": oracle_sample.single_core}
 
     if rank == 0:
         print(json.dumps(line))
