@@ -415,12 +415,18 @@ extern "C" int mcce_moe_forward(mcce_ctx* ctx, const void* hidden, const int32_t
   return MCCE_OK;
 }
 
+extern "C" int mcce_pipeline_wait(mcce_ctx* ctx);
+
 extern "C" int mcce_decode_step_host(mcce_ctx* ctx, const void* hidden_host, float* y_host, int32_t* sel_idx_host,
                                      void* cuda_stream) {
   if (!ctx || !hidden_host || !y_host) return MCCE_EINVAL;
   const mcce_config& c = ctx->cfg;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   const size_t LS = (size_t)c.n_layers * c.n_streams, esz = c.hidden_dtype == MCCE_BF16 ? 2 : 4;
+  {  // this call shares the first staging slot with the pipelined entry point: let its steps finish first
+    const int rcw = mcce_pipeline_wait(ctx);
+    if (rcw != MCCE_OK) return rcw;
+  }
   CK(cudaMemcpyAsync(ctx->stage_hidden, hidden_host, LS * c.d_model * esz, cudaMemcpyHostToDevice, st));
   int rc = mcce_route_step(ctx, 1, ctx->stage_hidden, nullptr, ctx->stage_sel, ctx->stage_w, nullptr, cuda_stream);
   if (rc != MCCE_OK) return rc;
