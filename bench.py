@@ -51,6 +51,9 @@ def parse_args():
     ap.add_argument("--max-rank", type=int, default=None, help="M of Max-Rank (default 2K)")
     ap.add_argument("--cum-p", type=float, default=0.5, help="p of Cumsum-Threshold")
     ap.add_argument("--lifetimes", action="store_true", help="also track and report cache lifetimes")
+    ap.add_argument("--chained", action="store_true",
+                    help="sequential-layer mode: the layers of a token chained through a residual stream (L rounds "
+                         "of single-layer launches per step) instead of independent layers")
     ap.add_argument("--impl", default="mcce", choices=["mcce", "reference"])
     ap.add_argument("--ffn", default="auto", choices=["auto", "simt", "tensor"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -254,6 +257,9 @@ def main_arm(args):
     y = torch.empty((wl.L, wl.S, wl.d), dtype=torch.float32, device=dev)
 
     def step(t):
+        if args.chained:
+            eng.decode_step_chained(hidden[t, 0])
+            return
         eng.route_step(hidden=hidden[t], out=(sel, sw))
         eng.moe_forward(hidden[t], sel[0], sw[0], out=y)
 
@@ -328,6 +334,7 @@ def main_arm(args):
             "config": config_of(wl, {"l2": "inputs larger than L2: %.1f GB of expert weights streamed per step"
                                            % ((bytes_up + bytes_down) / 1e9),
                                      "ffn_path": "tensor" if _uses_tensor(eng) else "simt",
+                                     "layer_mode": "chained through a residual stream" if args.chained else "independent",
                                      "rerank": args.rerank if args.rerank == "prior" else (
                                          "maxrank M=%d" % max_rank if args.rerank == "maxrank"
                                          else "cumsum p=%g" % args.cum_p),
@@ -338,7 +345,7 @@ def main_arm(args):
             "gpu_launches": K * 6, "clocks": clocks}
 
     # ---- routing alone, several tokens per launch (state stays in registers, the GEMM sees more tiles) -----
-    if not args.no_kernel_timing and wl.bf16 and n_tok >= 8:
+    if not args.no_kernel_timing and wl.bf16 and n_tok >= 8 and not args.chained:
         eng.profile(True)
         eng.profile_read(reset=True)
         sel8 = torch.empty((8, wl.L, wl.S, wl.K), dtype=torch.int32, device=dev)
@@ -361,7 +368,7 @@ def main_arm(args):
                                   "tokens_per_stream": n_tok}
 
     # ---- end to end through the host-buffer entry points ----------------------------------------------------
-    if not args.no_e2e:
+    if not args.no_e2e and not args.chained:
         n_e2e = max(4, min(K, 20))
         hh = torch.empty((n_e2e + 1, wl.L, wl.S, wl.d), dtype=wdt).pin_memory()
         hh.copy_(hidden[:n_e2e + 1])

@@ -134,6 +134,18 @@ int mcce_route_step(mcce_ctx* ctx, int32_t n_steps, const void* hidden, const fl
 int mcce_moe_forward(mcce_ctx* ctx, const void* hidden, const int32_t* sel_idx, const float* sel_w,
                      float* y, void* cuda_stream);
 
+/* One token in sequential-layer mode: the layers are chained through a residual stream instead of being
+ * independent, as in a real decoder (the paper changes nothing in the forward pass but the ranking, Sec. 2.2).
+ * For l = 0..L-1: route layer l on its input x_l, run its experts, x_{l+1} = x_l + y_l rounded to the hidden
+ * dtype (no normalisation layer: the logit scale may drift with depth, which the per-layer Delta_avg absorbs).
+ *   x0     DEVICE hidden_dtype [S,d]: input of layer 0        x_out DEVICE hidden_dtype [S,d]: output of layer L-1
+ *   sel_idx DEVICE int32 [L,S,K], optional: the selections of every layer
+ * Cache state, counters, Delta statistics and the miss trace advance exactly as with mcce_route_step.  Launches
+ * L rounds of the single-layer kernels on the stream (asynchronous).  On the tensor-core path the expert
+ * outputs are summed with fp32 atomics, so x_{l+1} can differ in its last bit between runs, and with it,
+ * rarely, a near-tie routing decision of a later layer. */
+int mcce_decode_step_chained(mcce_ctx* ctx, const void* x0, void* x_out, int32_t* sel_idx, void* cuda_stream);
+
 /* One whole decode step from HOST buffers: copies hidden [L,S,d] to the device, routes, runs the
  * experts and copies y [L,S,d] (and, if non-NULL, sel_idx [L,S,K]) back.  Staging lives in the
  * workspace.  hidden_host / y_host should be pinned.  Synchronises the stream before returning. */

@@ -22,7 +22,7 @@ RERANK_CACHE_PRIOR, RERANK_MAX_RANK, RERANK_CUMSUM = 0, 1, 2
 
 EXPORTS = [
     "mcce_workspace_bytes", "mcce_create", "mcce_destroy", "mcce_set_router", "mcce_set_experts", "mcce_reset",
-    "mcce_route_step", "mcce_moe_forward", "mcce_decode_step_host", "mcce_pipeline_submit_host", "mcce_pipeline_wait", "mcce_cache_stats", "mcce_get_cache_state",
+    "mcce_route_step", "mcce_moe_forward", "mcce_decode_step_host", "mcce_decode_step_chained", "mcce_pipeline_submit_host", "mcce_pipeline_wait", "mcce_cache_stats", "mcce_get_cache_state",
     "mcce_get_grouping", "mcce_lifetime_stats", "mcce_set_miss_trace", "mcce_belady_replay", "mcce_profile", "mcce_profile_read", "mcce_uses_tensor_path", "mcce_selftest_wait_timeout", "mcce_route_trace_static",
     "mcce_route_trace_static_limit", "mcce_gen_normal", "mcce_gen_hidden_step", "mcce_gen_philox_words", "mcce_strerror",
     "mcce_last_cuda_error",
@@ -70,6 +70,7 @@ def load():
         lib.mcce_route_step.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp]
         lib.mcce_moe_forward.argtypes = [vp] * 6
         lib.mcce_decode_step_host.argtypes = [vp] * 5
+        lib.mcce_decode_step_chained.argtypes = [vp] * 5
         lib.mcce_pipeline_submit_host.argtypes = [vp] * 5
         lib.mcce_pipeline_wait.argtypes = [vp]
         lib.mcce_cache_stats.argtypes = [vp, C.POINTER(Stats), C.POINTER(Stats)]
@@ -210,6 +211,14 @@ class Engine:
         assert not hidden_host.is_cuda and not y_host.is_cuda
         _check(self.lib.mcce_decode_step_host(self.ctx, _ptr(hidden_host), _ptr(y_host), _ptr(sel_host), _stream()),
                self.ctx)
+
+    def decode_step_chained(self, x0: torch.Tensor, want_sel=False):
+        """One token with the layers chained through a residual stream: x0 [S,d] -> x_L [S,d] (and sel [L,S,K])."""
+        assert x0.dtype == _tdtype(self.dtype) and x0.numel() == self.S * self.d
+        x_out = torch.empty_like(x0)
+        sel = torch.empty((self.L, self.S, self.K), dtype=torch.int32, device=self.device) if want_sel else None
+        _check(self.lib.mcce_decode_step_chained(self.ctx, _ptr(x0), _ptr(x_out), _ptr(sel), _stream()), self.ctx)
+        return (x_out, sel) if want_sel else x_out
 
     def pipeline_submit_host(self, hidden_host, y_host, sel_host=None):
         """Asynchronous variant of decode_step_host: copies overlap the compute of neighbouring steps; call

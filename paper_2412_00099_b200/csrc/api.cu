@@ -185,7 +185,7 @@ int timed(mcce_ctx* ctx, int kind, cudaStream_t st, F launch) {
 FfnParams ffn_params(const mcce_ctx* ctx, const void* hidden, const float* sel_w, float* y) {
   const mcce_config& c = ctx->cfg;
   FfnParams f;
-  f.L = c.n_layers, f.S = c.n_streams, f.E = c.n_experts, f.K = c.top_k, f.n_sh = c.n_shared;
+  f.L = c.n_layers, f.S = c.n_streams, f.E = c.n_experts, f.K = c.top_k, f.n_sh = c.n_shared, f.l0 = 0;
   f.d = c.d_model, f.I = c.d_ff, f.bf16 = c.hidden_dtype == MCCE_BF16;
   f.hidden = hidden;
   f.Wg = ctx->Wg, f.Wu = ctx->Wu, f.Wd = ctx->Wd, f.shWg = ctx->shWg, f.shWu = ctx->shWu, f.shWd = ctx->shWd;
@@ -390,18 +390,18 @@ extern "C" int mcce_route_step(mcce_ctx* ctx, int32_t n_steps, const void* hidde
   return MCCE_OK;
 }
 
-extern "C" int mcce_moe_forward(mcce_ctx* ctx, const void* hidden, const int32_t* sel_idx, const float* sel_w,
-                                float* y, void* cuda_stream) {
-  if (!ctx || !hidden || !sel_idx || !sel_w || !y) return MCCE_EINVAL;
-  if (!ctx->Wg) return MCCE_ESTATE;
-  if (((uintptr_t)hidden % 16) || ((uintptr_t)y % 16)) return MCCE_EINVAL;
+// Expert forward for model layers [l0, l0 + Ls): hidden, sel_idx, sel_w and y hold those layers only.  The
+// grouping, gathered rows and intermediates use the front of the context's buffers; only the expert weights
+// are addressed by model layer.
+static int forward_layers(mcce_ctx* ctx, int l0, int Ls, const void* hidden, const int32_t* sel_idx,
+                          const float* sel_w, float* y, cudaStream_t st) {
   const mcce_config& c = ctx->cfg;
-  cudaStream_t st = (cudaStream_t)cuda_stream;
   GroupParams g;
-  g.L = c.n_layers, g.S = c.n_streams, g.E = c.n_experts, g.K = c.top_k;
+  g.L = Ls, g.S = c.n_streams, g.E = c.n_experts, g.K = c.top_k;
   g.sel_idx = sel_idx, g.offsets = ctx->offsets, g.perm = ctx->perm, g.inv = ctx->inv;
   TIMED(MCCE_K_GROUP, st, launch_group(g, st));
-  const FfnParams f = ffn_params(ctx, hidden, sel_w, y);
+  FfnParams f = ffn_params(ctx, hidden, sel_w, y);
+  f.L = Ls, f.l0 = l0;
   // on the tensor path the down kernel adds w * E_i(x) into y itself: the gather pass clears y on the way
   TIMED(MCCE_K_GATHER, st, launch_gather(f, ctx->use_tc != 0, st));
   if (ctx->use_tc) {
@@ -415,7 +415,85 @@ extern "C" int mcce_moe_forward(mcce_ctx* ctx, const void* hidden, const int32_t
   return MCCE_OK;
 }
 
+extern "C" int mcce_moe_forward(mcce_ctx* ctx, const void* hidden, const int32_t* sel_idx, const float* sel_w,
+                                float* y, void* cuda_stream) {
+  if (!ctx || !hidden || !sel_idx || !sel_w || !y) return MCCE_EINVAL;
+  if (!ctx->Wg) return MCCE_ESTATE;
+  if (((uintptr_t)hidden % 16) || ((uintptr_t)y % 16)) return MCCE_EINVAL;
+  return forward_layers(ctx, 0, ctx->cfg.n_layers, hidden, sel_idx, sel_w, y, (cudaStream_t)cuda_stream);
+}
+
 extern "C" int mcce_pipeline_wait(mcce_ctx* ctx);
+
+// ---- sequential-layer mode: the layers of one token chained through a residual stream --------------------
+// Routing of model layer l from its input x [S,d]: the same kernels as mcce_route_step, launched for one layer.
+static int route_one_layer(mcce_ctx* ctx, int l, const void* x, int32_t* sel, float* w, cudaStream_t st) {
+  const mcce_config& c = ctx->cfg;
+  const size_t S = c.n_streams, E = c.n_experts, EW = ctx->EW;
+  RouteParams p;
+  p.L = 1, p.S = c.n_streams, p.E = c.n_experts, p.K = c.top_k, p.J = c.top_j, p.C = c.cache_capacity;
+  p.d = c.d_model, p.n_steps = 1, p.lambda = c.lambda, p.delta_mode = c.delta_mode, p.renorm = c.renorm;
+  p.rerank_mode = c.rerank_mode, p.max_rank = c.max_rank, p.cum_threshold = c.cum_threshold;
+  p.hidden_bf16 = c.hidden_dtype == MCCE_BF16;
+  p.Wr = ctx->Wr + (size_t)l * E * c.d_model;
+  p.fixed_delta = ctx->fixed_delta ? ctx->fixed_delta + l : nullptr;
+  p.stamp = ctx->stamp + (size_t)l * S * E, p.ever = ctx->ever + (size_t)l * S * EW;
+  p.sum_range = ctx->sum_range + (size_t)l * S, p.miss = ctx->miss + (size_t)l * S, p.cold = ctx->cold + (size_t)l * S;
+  p.load_tok = ctx->load_tok ? ctx->load_tok + (size_t)l * S * E : nullptr;
+  p.life = ctx->life ? ctx->life + (size_t)l * S * 3 : nullptr;
+  const bool trace = ctx->miss_trace && ctx->trace_pos < ctx->trace_cap;
+  p.miss_trace = trace ? ctx->miss_trace + ((size_t)ctx->trace_pos * c.n_layers + l) * S : nullptr;
+  p.trace_avail = trace ? 1 : 0;
+  p.sel_idx = sel, p.sel_w = w, p.logits_out = nullptr;
+  p.tok0 = (uint32_t)ctx->tok, p.cnt0 = (uint32_t)ctx->delta_cnt;
+  if (ctx->use_tc_router && ctx->rg.ready) {
+    int ks = 1;
+    TIMED(MCCE_K_ROUTE_GEMM, st, router_gemm_launch(ctx->rg, c, x, 1, ctx->z_buf, &ks, ctx->err, st, l, 1));
+    p.hidden = nullptr, p.logits_in = ctx->z_buf, p.n_partials = ks, p.partial_stride = S * E;
+  } else {
+    p.hidden = x, p.logits_in = nullptr, p.n_partials = 1, p.partial_stride = 0;
+  }
+  TIMED(MCCE_K_ROUTE, st, launch_route(p, st));
+  return MCCE_OK;
+}
+
+extern "C" int mcce_decode_step_chained(mcce_ctx* ctx, const void* x0, void* x_out, int32_t* sel_idx,
+                                        void* cuda_stream) {
+  if (!ctx || !x0 || !x_out) return MCCE_EINVAL;
+  if (!ctx->Wr || !ctx->Wg) return MCCE_ESTATE;
+  if (((uintptr_t)x0 % 16) || ((uintptr_t)x_out % 16)) return MCCE_EINVAL;
+  const mcce_config& c = ctx->cfg;
+  if (c.delta_mode == MCCE_DELTA_FIXED && !ctx->fixed_delta) return MCCE_ESTATE;
+  const uint64_t last_key = (uint64_t)c.n_experts + (ctx->tok + 1) * (uint64_t)c.top_k + c.top_k + 1;
+  if (last_key >= 0xffffffffull || ctx->delta_cnt + 1 >= 0xffffffffull) return MCCE_ESTATE;
+  {
+    const int rcw = mcce_pipeline_wait(ctx);   // the staging buffers are used as the residual stream
+    if (rcw != MCCE_OK) return rcw;
+  }
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  const size_t S = c.n_streams, K = c.top_k, n = S * c.d_model;
+  const bool bf16 = c.hidden_dtype == MCCE_BF16;
+  void* buf[2] = {ctx->stage_hidden, ctx->stage_hidden2};
+  const void* x = x0;
+  for (int l = 0; l < c.n_layers; ++l) {
+    int32_t* sel = ctx->stage_sel + (size_t)l * S * K;
+    float* w = ctx->stage_w + (size_t)l * S * K;
+    int rc = route_one_layer(ctx, l, x, sel, w, st);
+    if (rc != MCCE_OK) return rc;
+    rc = forward_layers(ctx, l, 1, x, sel, w, ctx->stage_y, st);
+    if (rc != MCCE_OK) return rc;
+    void* nxt = l + 1 == c.n_layers ? x_out : buf[l & 1];
+    CK(launch_residual(x, ctx->stage_y, nxt, n, bf16, st));
+    x = nxt;
+  }
+  if (sel_idx)
+    CK(cudaMemcpyAsync(sel_idx, ctx->stage_sel, (size_t)c.n_layers * S * K * 4, cudaMemcpyDeviceToDevice, st));
+  ctx->tok += 1;
+  ctx->steps_since_reset += 1;
+  if (ctx->miss_trace) ctx->trace_pos += 1;
+  if (c.delta_mode == MCCE_DELTA_RUNNING) ctx->delta_cnt += 1;
+  return MCCE_OK;
+}
 
 extern "C" int mcce_decode_step_host(mcce_ctx* ctx, const void* hidden_host, float* y_host, int32_t* sel_idx_host,
                                      void* cuda_stream) {

@@ -56,6 +56,7 @@ struct GroupParams {
 // shared experts, [l][q][s].
 struct FfnParams {
   int L, S, E, K, n_sh, d, I;
+  int l0;  // model layer of local layer 0: only the weights are indexed by model layer, everything else is local
   int bf16;
   const void* hidden;  // [L,S,d]
   const void *Wg, *Wu, *Wd, *shWg, *shWu, *shWd;
@@ -80,7 +81,7 @@ bool router_gemm_applicable(const mcce_config& c);
 int router_gemm_steps_max();
 int router_gemm_plan(const mcce_config& c, const float* Wr, void* terms, RouterGemmPlan* plan, cudaStream_t st);
 cudaError_t router_gemm_launch(RouterGemmPlan& plan, const mcce_config& c, const void* hidden, int n_steps, float* Z,
-                               int* k_split, uint32_t* err, cudaStream_t st);
+                               int* k_split, uint32_t* err, cudaStream_t st, int l0 = 0, int n_layers = 0);
 
 cudaError_t launch_wait_timeout_selftest(uint32_t* err, unsigned long long limit_ns, uint32_t* outcome,
                                          cudaStream_t st);
@@ -90,6 +91,7 @@ cudaError_t launch_gather(const FfnParams& p, bool zero_y, cudaStream_t st);
 cudaError_t launch_ffn_simt_up(const FfnParams& p, cudaStream_t st);
 cudaError_t launch_ffn_simt_down(const FfnParams& p, cudaStream_t st);
 cudaError_t launch_combine(const FfnParams& p, cudaStream_t st);
+cudaError_t launch_residual(const void* x_in, const float* y, void* x_out, size_t n, bool bf16, cudaStream_t st);
 cudaError_t launch_stats(const uint32_t* miss, const uint32_t* cold, unsigned long long* out, int L, int S,
                          cudaStream_t st);
 

@@ -51,7 +51,7 @@ __global__ void __launch_bounds__(kTB * 32) ffn_simt_kernel(const FfnParams p) {
     const int o0 = p.offsets[(size_t)l * (p.E + 1) + e], o1 = p.offsets[(size_t)l * (p.E + 1) + e + 1];
     row0 = (size_t)l * P + o0;
     m = o1 - o0;
-    const size_t wi = (size_t)l * p.E + e;
+    const size_t wi = (size_t)(p.l0 + l) * p.E + e;
     if (GATE_UP) {
       in = (const T*)p.Xg + row0 * p.d;
       W0 = (const T*)p.Wg + wi * wsz;
@@ -64,7 +64,7 @@ __global__ void __launch_bounds__(kTB * 32) ffn_simt_kernel(const FfnParams p) {
     const int q = e - p.E;
     row0 = (size_t)p.L * P + ((size_t)l * p.n_sh + q) * p.S;
     m = p.S;
-    const size_t wi = (size_t)l * p.n_sh + q;
+    const size_t wi = (size_t)(p.l0 + l) * p.n_sh + q;
     if (GATE_UP) {
       in = (const T*)p.hidden + (size_t)l * p.S * p.d;
       W0 = (const T*)p.shWg + wi * wsz;

@@ -50,6 +50,7 @@ struct Cfg {
 
 struct TcArgs {
   int L, S, E, K, n_sh, d, I;
+  int l0;                // model layer of local layer 0 (weights are indexed by model layer)
   int n_items;
   const int32_t* offsets;
   const int32_t* perm;   // [L, S*K] position -> pair, for the fused combine of the down kernel
@@ -99,7 +100,7 @@ __device__ __forceinline__ Item decode(const TcArgs& a, int w) {
     const int o0 = __ldg(a.offsets + (size_t)l * (a.E + 1) + g);
     it.m = __ldg(a.offsets + (size_t)l * (a.E + 1) + g + 1) - o0;
     it.shared = false;
-    it.wrow = (l * a.E + g) * rows + it.col0;
+    it.wrow = ((a.l0 + l) * a.E + g) * rows + it.col0;
     it.xrow = l * P + o0;
     it.orow = (size_t)it.xrow;
   } else {
@@ -108,7 +109,7 @@ __device__ __forceinline__ Item decode(const TcArgs& a, int w) {
     it.col0 = rt * span;
     it.m = min(kNMax, a.S - c * kNMax);
     it.shared = true;
-    it.wrow = (l * a.n_sh + q) * rows + it.col0;
+    it.wrow = ((a.l0 + l) * a.n_sh + q) * rows + it.col0;
     it.orow = (size_t)a.L * P + (size_t)(l * a.n_sh + q) * a.S + c * kNMax;
     it.xrow = UP ? l * a.S + c * kNMax : (int)it.orow;   // up: rows of the hidden tensor; down: rows of H
   }
@@ -333,7 +334,7 @@ cudaError_t launch(const TcMaps& maps, const FfnParams& p, uint32_t* err, cudaSt
   cudaError_t e0 = sm_count_and_smem_optin(ffn_tc_kernel<UP>, Cfg<UP>::kSmemBytes, cache, &sms);
   if (e0 != cudaSuccess) return e0;
   TcArgs a;
-  a.L = p.L, a.S = p.S, a.E = p.E, a.K = p.K, a.n_sh = p.n_sh, a.d = p.d, a.I = p.I;
+  a.L = p.L, a.S = p.S, a.E = p.E, a.K = p.K, a.n_sh = p.n_sh, a.d = p.d, a.I = p.I, a.l0 = p.l0;
   a.n_items = p.L * items_per_layer(p.E, p.n_sh, p.S, UP ? p.I / kTileM : (p.d / kTileM + 1) / 2);
   a.offsets = p.offsets, a.perm = p.perm, a.sel_w = p.sel_w, a.H = (__nv_bfloat16*)p.H, a.y = p.y, a.err = err;
   const int grid = a.n_items < sms ? a.n_items : sms;
@@ -360,15 +361,17 @@ int tc_plan(const mcce_config& c, const void* Wg, const void* Wu, const void* Wd
          make_map(&plan->sh_up, shWu, L * nsh * I, d, kTileM) && make_map(&plan->sh_down, shWd, L * nsh * d, I, kTileM);
   ok = ok && make_map(&plan->x_routed, Xg, L * S * K + 256, d, kXBox) && make_map(&plan->h_all, H, rows + 256, I, kXBox);
   plan->hidden_ptr = nullptr;
+  plan->hidden_rows = 0;
   plan->ready = ok;
   return ok ? MCCE_OK : MCCE_ECUDA;
 }
 
 cudaError_t tc_launch_up(TcPlan& plan, const FfnParams& p, uint32_t* err_flag, cudaStream_t st) {
   if (!plan.ready) return cudaErrorNotReady;
-  if (p.n_sh && plan.hidden_ptr != p.hidden) {
+  if (p.n_sh && (plan.hidden_ptr != p.hidden || plan.hidden_rows != (uint64_t)p.L * p.S)) {
     if (!make_map(&plan.x_hidden, p.hidden, (uint64_t)p.L * p.S, p.d, kXBox)) return cudaErrorInvalidValue;
     plan.hidden_ptr = p.hidden;
+    plan.hidden_rows = (uint64_t)p.L * p.S;
   }
   TcMaps m;
   m.w0 = plan.w_gate, m.w1 = plan.w_up, m.x = plan.x_routed;

@@ -12,6 +12,7 @@ struct TcPlan {
   alignas(64) CUtensorMap w_gate, w_up, w_down, sh_gate, sh_up, sh_down;  // weights, 128-row boxes
   alignas(64) CUtensorMap x_routed, x_hidden, h_all;                      // activations, 16-row boxes
   const void* hidden_ptr;   // the hidden tensor x_hidden was built for
+  uint64_t hidden_rows;     // and its row count
   int ready;
 };
 

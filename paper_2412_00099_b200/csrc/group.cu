@@ -102,4 +102,22 @@ cudaError_t launch_gather(const FfnParams& p, bool zero_y, cudaStream_t st) {
   return cudaGetLastError();
 }
 
+// Residual stream of the sequential-layer mode: x_out = x_in + y, rounded to the hidden dtype.
+__global__ void residual_kernel(const void* x_in, const float* y, void* x_out, size_t n, int bf16) {
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+    if (bf16) {
+      const float v = __fadd_rn(__bfloat162float(((const __nv_bfloat16*)x_in)[i]), y[i]);
+      ((__nv_bfloat16*)x_out)[i] = __float2bfloat16_rn(v);
+    } else {
+      ((float*)x_out)[i] = __fadd_rn(((const float*)x_in)[i], y[i]);
+    }
+  }
+}
+
+cudaError_t launch_residual(const void* x_in, const float* y, void* x_out, size_t n, bool bf16, cudaStream_t st) {
+  const unsigned grid = (unsigned)((n + 255) / 256 > 2048 ? 2048 : (n + 255) / 256);
+  residual_kernel<<<grid, 256, 0, st>>>(x_in, y, x_out, n, bf16 ? 1 : 0);
+  return cudaGetLastError();
+}
+
 }  // namespace mcce

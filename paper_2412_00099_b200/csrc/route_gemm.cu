@@ -44,6 +44,7 @@ constexpr size_t kSmemBytes = (size_t)kRingBytes + 1024 + 256;
 
 struct GemmArgs {
   int L, S, E, d, n_steps, NS;
+  int l0, L_terms; // first layer of this launch; layers in the term tensor (stride between the three terms)
   int RA;          // router rows per term tile actually loaded
   int KS, kt_per;  // K-split: partial sums over kt_per slabs each
   int n_stages;
@@ -134,7 +135,7 @@ router_gemm_kernel(const __grid_constant__ GemmMaps maps, const GemmArgs a) {
           mbar_expect_tx(full, tx);
 #pragma unroll
           for (int p = 0; p < 3; ++p)
-            tma_load_3d(sa + p * kABytes, &maps.w, kt * kTileK, it.mt * kTileM, p * a.L + it.l, full);
+            tma_load_3d(sa + p * kABytes, &maps.w, kt * kTileK, it.mt * kTileM, p * a.L_terms + a.l0 + it.l, full);
           const uint32_t sb = sa + 3 * kABytes;
           for (int j = 0; j < a.NS; j += kXBox)
             tma_load_2d(sb + j * kTileK * 2, &maps.x, kt * kTileK, it.row0 + j, full);
@@ -301,12 +302,13 @@ int router_gemm_plan(const mcce_config& c, const float* Wr, void* terms, RouterG
 }
 
 cudaError_t router_gemm_launch(RouterGemmPlan& plan, const mcce_config& c, const void* hidden, int n_steps, float* Z,
-                               int* k_split, uint32_t* err, cudaStream_t st) {
+                               int* k_split, uint32_t* err, cudaStream_t st, int l0, int n_layers) {
+  const int Ls = n_layers > 0 ? n_layers : c.n_layers;   // layers [l0, l0 + Ls) of the model; hidden holds those only
   static int cache[64] = {0};
   int sms = 0;
   cudaError_t e0 = sm_count_and_smem_optin(router_gemm_kernel, kSmemBytes, cache, &sms);
   if (e0 != cudaSuccess) return e0;
-  const uint64_t rows = (uint64_t)n_steps * c.n_layers * c.n_streams;
+  const uint64_t rows = (uint64_t)n_steps * Ls * c.n_streams;
   if (plan.hidden_ptr != hidden || plan.hidden_rows != rows) {
     EncodeFn fn = encode_fn();
     const cuuint64_t dims[2] = {(cuuint64_t)c.d_model, rows};
@@ -321,7 +323,8 @@ cudaError_t router_gemm_launch(RouterGemmPlan& plan, const mcce_config& c, const
     plan.hidden_rows = rows;
   }
   GemmArgs a;
-  a.L = c.n_layers, a.S = c.n_streams, a.E = c.n_experts, a.d = c.d_model, a.n_steps = n_steps;
+  a.L = Ls, a.S = c.n_streams, a.E = c.n_experts, a.d = c.d_model, a.n_steps = n_steps;
+  a.l0 = l0, a.L_terms = c.n_layers;
   // streams per tile: as many as TMEM holds; narrower only when even the deepest K-split would leave most SMs idle
   int ns = c.n_streams >= kNSMax ? kNSMax : (c.n_streams + 15) & ~15;
   const int mt = (c.n_experts + kTileM - 1) / kTileM;
@@ -329,12 +332,12 @@ cudaError_t router_gemm_launch(RouterGemmPlan& plan, const mcce_config& c, const
   int ks_max = 1;
   while (ks_max < 8 && kt % (2 * ks_max) == 0 && kt / (2 * ks_max) >= 4 && n_steps * 2 * ks_max <= router_gemm_steps_max())
     ks_max *= 2;
-  while (ns > 16 && n_steps * c.n_layers * mt * ((c.n_streams + ns - 1) / ns) * ks_max < sms / 2) ns /= 2;
+  while (ns > 16 && n_steps * Ls * mt * ((c.n_streams + ns - 1) / ns) * ks_max < sms / 2) ns /= 2;
   ns = (ns + 15) & ~15;
   a.NS = ns;
   // split the reduction over up to eight CTAs per tile while SMs would otherwise idle; the partial
   // logits are summed by the routing tail.  The logits buffer has router_gemm_steps_max() slots.
-  const int items = n_steps * c.n_layers * mt * ((c.n_streams + ns - 1) / ns);
+  const int items = n_steps * Ls * mt * ((c.n_streams + ns - 1) / ns);
   // Cost of a split, from measurements on B200: a round of the persistent grid costs about 1 us per K-slab
   // of its items (twelve MMAs) plus about 5 us of fill and drain, so one round of shorter items wins.
   int ks = 1;
