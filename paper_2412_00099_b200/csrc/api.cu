@@ -127,7 +127,9 @@ Layout layout_of(const mcce_config& c) {
   o.st_y2 = take(L * S * d * 4);
   const bool rg = router_gemm_applicable(c);
   o.wr_terms = take(rg ? 3 * L * E * d * 2 : 0);
-  o.z_buf = take(rg ? (size_t)router_gemm_steps_max() * L * S * E * 4 : 0);
+  // logits of up to router_gemm_steps_max() tokens; the router-resident kernel writes one array per K part
+  const size_t z_slots = (size_t)router_gemm_steps_max() * (router_gemm_res_applicable(c) ? router_gemm_res_parts_max() : 1);
+  o.z_buf = take(rg ? z_slots * L * S * E * 4 : 0);
   o.load_tok = take(c.track_lifetime ? L * S * E * 4 : 0);
   o.life = take(c.track_lifetime ? L * S * 3 * 8 : 0);
   o.total = p;
@@ -270,6 +272,10 @@ extern "C" int mcce_set_router(mcce_ctx* ctx, const float* Wr, const float* fixe
     CK(cudaSetDevice(ctx->cfg.device));
     const int rc = router_gemm_plan(ctx->cfg, Wr, ctx->wr_terms, &ctx->rg, 0);
     if (rc != MCCE_OK) return rc;
+    if (router_gemm_res_applicable(ctx->cfg)) {
+      const int rc2 = router_gemm_res_plan(ctx->cfg, ctx->wr_terms, &ctx->rg);
+      if (rc2 != MCCE_OK) return rc2;
+    }
     CK(cudaDeviceSynchronize());
   }
   return MCCE_OK;
@@ -367,7 +373,12 @@ extern "C" int mcce_route_step(mcce_ctx* ctx, int32_t n_steps, const void* hidde
       const int nt = n_steps - t0 < router_gemm_steps_max() ? n_steps - t0 : router_gemm_steps_max();
       const char* h = (const char*)hidden + (size_t)t0 * LS * c.d_model * esz;
       int ks = 1;
-      TIMED(MCCE_K_ROUTE_GEMM, st, router_gemm_launch(ctx->rg, c, h, nt, ctx->z_buf, &ks, ctx->err, st));
+      if (ctx->rg.res_ready) {
+        ks = ctx->rg.res_parts;
+        TIMED(MCCE_K_ROUTE_GEMM, st, router_gemm_res_launch(ctx->rg, c, h, nt, ctx->z_buf, ctx->err, st));
+      } else {
+        TIMED(MCCE_K_ROUTE_GEMM, st, router_gemm_launch(ctx->rg, c, h, nt, ctx->z_buf, &ks, ctx->err, st));
+      }
       p.n_steps = nt, p.hidden = nullptr, p.logits_in = ctx->z_buf;
       p.n_partials = ks, p.partial_stride = (size_t)nt * LS * c.n_experts;
       p.sel_idx = sel_idx + (size_t)t0 * LS * c.top_k, p.sel_w = sel_w + (size_t)t0 * LS * c.top_k;

@@ -73,15 +73,25 @@ struct FfnParams {
 // Router logits on the tensor cores (route_gemm.cu).  Plain data: lives inside the zero-initialised context.
 struct RouterGemmPlan {
   alignas(64) CUtensorMap w, x;
+  alignas(64) CUtensorMap w_res, x_res, xt_res;   // router-resident kernel (route_gemm_res.cu)
   const void* hidden_ptr;
   uint64_t hidden_rows;
+  const void* hidden_ptr_res;
+  uint64_t hidden_rows_res;
   int ready;
+  int res_ready, res_parts;   // K parts (= partial logit arrays) of the router-resident kernel
 };
 bool router_gemm_applicable(const mcce_config& c);
 int router_gemm_steps_max();
 int router_gemm_plan(const mcce_config& c, const float* Wr, void* terms, RouterGemmPlan* plan, cudaStream_t st);
 cudaError_t router_gemm_launch(RouterGemmPlan& plan, const mcce_config& c, const void* hidden, int n_steps, float* Z,
                                int* k_split, uint32_t* err, cudaStream_t st, int l0 = 0, int n_layers = 0);
+
+bool router_gemm_res_applicable(const mcce_config& c);
+int router_gemm_res_parts_max();
+int router_gemm_res_plan(const mcce_config& c, void* terms, RouterGemmPlan* plan);
+cudaError_t router_gemm_res_launch(RouterGemmPlan& plan, const mcce_config& c, const void* hidden, int n_steps,
+                                   float* Z, uint32_t* err, cudaStream_t st);
 
 cudaError_t launch_wait_timeout_selftest(uint32_t* err, unsigned long long limit_ns, uint32_t* outcome,
                                          cudaStream_t st);
