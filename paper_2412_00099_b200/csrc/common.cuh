@@ -95,7 +95,9 @@ cudaError_t router_gemm_res_launch(RouterGemmPlan& plan, const mcce_config& c, c
 
 cudaError_t launch_wait_timeout_selftest(uint32_t* err, unsigned long long limit_ns, uint32_t* outcome,
                                          cudaStream_t st);
-cudaError_t launch_route(const RouteParams& p, cudaStream_t st);
+cudaError_t launch_route(const RouteParams& p, cudaStream_t st);   // picks the thread-per-stream kernel where it applies
+bool route_thread_applicable(const RouteParams& p);
+cudaError_t launch_route_thread(const RouteParams& p, cudaStream_t st);
 cudaError_t launch_group(const GroupParams& p, cudaStream_t st);
 cudaError_t launch_gather(const FfnParams& p, bool zero_y, cudaStream_t st);
 cudaError_t launch_ffn_simt_up(const FfnParams& p, cudaStream_t st);

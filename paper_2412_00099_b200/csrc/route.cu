@@ -366,6 +366,7 @@ static cudaError_t launch_ne(const RouteParams& p, cudaStream_t st) {
 }
 
 cudaError_t launch_route(const RouteParams& p, cudaStream_t st) {
+  if (route_thread_applicable(p)) return launch_route_thread(p, st);
   const int ne = (p.E + 31) / 32;
   if (ne <= 1) return launch_ne<1>(p, st);
   if (ne <= 2) return launch_ne<2>(p, st);

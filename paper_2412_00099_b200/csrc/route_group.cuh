@@ -1,0 +1,363 @@
+// Routing tail of a small group of lanes per (stream, layer): the device code shared by the stand-alone
+// kernel (route_thread.cu) and the kernel that runs it beside the router GEMM (route_fused.cu).
+//
+// A stream belongs to G = N/8 adjacent lanes (N = experts rounded up to 8, 16, 32 or 64), each holding eight
+// consecutive experts as order-preserving integer keys in registers: a selection is a comparison tree over the
+// lane's own eight keys followed by log2(G) butterfly steps inside the group; several streams advance per warp
+// instruction.  Recency keys, resident and ever-resident bits stay in registers across the tokens of a launch.
+// The state arrays in global memory have the format of route.cu.  Decision arithmetic is the same single IEEE
+// fp32 operations in the same order as in route.cu (Eq. 7, Eq. 8, Eq. 4, Sec. 3.3, Sec. 4.2 of the paper).
+#pragma once
+#include "common.cuh"
+#include "warp_select.cuh"
+
+namespace mcce {
+namespace rgroup {
+
+
+constexpr int kNE = 8;        // experts per lane
+constexpr int kPartsMax = 8;  // partial logit arrays that the prefetch holds in registers
+
+struct Cand {
+  uint32_t k;   // selection key (0 = none)
+  int e;        // expert
+  uint32_t z;   // key of its unmodified logit
+};
+
+// better(a, b): b replaces a when its key is larger, or equal with the lower expert index
+__device__ __forceinline__ Cand pick(const Cand a, const Cand b) {
+  const bool c = b.k > a.k || (b.k == a.k && b.e < a.e);
+  Cand r;
+  r.k = c ? b.k : a.k, r.e = c ? b.e : a.e, r.z = c ? b.z : a.z;
+  return r;
+}
+
+// Largest key among the experts of the group not in `taken` (bit i = this lane's i-th expert); equal keys ->
+// lowest expert.  Every lane of the group gets the result.
+template <int G>
+__device__ __forceinline__ Cand group_argmax(const uint32_t (&key)[kNE], const uint32_t (&zk)[kNE], uint32_t taken, int e0) {
+  Cand c[kNE];
+#pragma unroll
+  for (int i = 0; i < kNE; ++i) c[i].k = ((taken >> i) & 1u) ? 0u : key[i], c[i].e = e0 + i, c[i].z = zk[i];
+#pragma unroll
+  for (int w = kNE / 2; w >= 1; w /= 2)
+#pragma unroll
+    for (int j = 0; j < w; ++j) {
+      // strict comparison: on equal keys the lower expert (left) stays
+      const bool gt = c[2 * j + 1].k > c[2 * j].k;
+      c[j].k = gt ? c[2 * j + 1].k : c[2 * j].k;
+      c[j].e = gt ? c[2 * j + 1].e : c[2 * j].e;
+      c[j].z = gt ? c[2 * j + 1].z : c[2 * j].z;
+    }
+  Cand best = c[0];
+  // butterfly inside the group (redux.sync restricted to the group's lanes was measured 40 % slower)
+#pragma unroll
+  for (int o = 1; o < G; o <<= 1) {
+    Cand other;
+    other.k = __shfl_xor_sync(kFull, best.k, o);
+    other.e = __shfl_xor_sync(kFull, best.e, o);
+    other.z = __shfl_xor_sync(kFull, best.z, o);
+    best = pick(best, other);
+  }
+  return best;
+}
+
+template <int G>
+__device__ __forceinline__ uint32_t group_max(uint32_t v) {
+#pragma unroll
+  for (int o = 1; o < G; o <<= 1) v = max(v, __shfl_xor_sync(kFull, v, o));
+  return v;
+}
+template <int G>
+__device__ __forceinline__ uint32_t group_min(uint32_t v) {
+#pragma unroll
+  for (int o = 1; o < G; o <<= 1) v = min(v, __shfl_xor_sync(kFull, v, o));
+  return v;
+}
+template <int G>
+__device__ __forceinline__ uint32_t group_or(uint32_t v) {
+#pragma unroll
+  for (int o = 1; o < G; o <<= 1) v |= __shfl_xor_sync(kFull, v, o);
+  return v;
+}
+template <int G>
+__device__ __forceinline__ float group_sum(float v) {
+#pragma unroll
+  for (int o = 1; o < G; o <<= 1) v += __shfl_xor_sync(kFull, v, o);
+  return v;
+}
+
+
+// Loads of logits: through the read-only path when another kernel wrote them, L2-coherent when CTAs of the
+// running kernel did.
+template <bool COHERENT>
+__device__ __forceinline__ float4 ldz4(const float4* q) { return COHERENT ? __ldcg(q) : __ldg(q); }
+template <bool COHERENT>
+__device__ __forceinline__ float ldz1(const float* q) { return COHERENT ? __ldcg(q) : __ldg(q); }
+
+// Routes the p.n_steps tokens of stream s_raw of layer l.  All 32 lanes of a warp must call this together
+// (groups past the last stream run on stream 0's data and store nothing).  `sub` is the lane's index in its
+// group.  wait(t) is called by every lane before the logits of token t are read and returns false to give up.
+template <int G, int KMAX, bool PF, bool COHERENT, typename Wait>
+__device__ __forceinline__ void route_group_streams(const RouteParams& p, const int l, const int s_raw, const int sub,
+                                                    Wait wait) {
+  // a group past the last stream runs on stream 0's data and stores nothing (its lanes share warps with live groups)
+  const bool active = s_raw < p.S;
+  const int s = active ? s_raw : 0;
+  const size_t pair = (size_t)l * p.S + s;
+  const int E = p.E, K = p.K;
+  const int e0 = sub * kNE;
+  const bool vec4 = (E & 3) == 0;
+
+  // ---- state of this (layer, stream) into registers -----------------------------------------------------
+  uint32_t st[kNE];
+  uint32_t resb = 0u, everb = 0u;   // bit i: this lane's i-th expert is resident / was ever resident
+  {
+    const int EW = (E + 31) >> 5;
+    const uint32_t word = e0 < E ? p.ever[pair * EW + (e0 >> 5)] : 0u;
+    everb = (word >> (e0 & 31)) & 0xffu;
+  }
+#pragma unroll
+  for (int i = 0; i < kNE; ++i) {
+    st[i] = e0 + i < E ? p.stamp[pair * E + e0 + i] : 0u;
+    resb |= (st[i] != 0u ? 1u : 0u) << i;
+  }
+  int resident = (int)group_sum<G>((float)__popc(resb));   // exact: at most 64
+  float sum_range = p.sum_range[pair];
+  uint32_t miss_c = p.miss[pair], cold_c = p.cold[pair];
+
+  // The partial logits of the next token are requested before the current token is routed, so that their
+  // latency (L2, mostly) is off the critical path: up to kPartsMax parts of eight logits per lane in flight.
+  const bool prefetch = PF;   // the launcher checks: rows 16-byte aligned, at most kPartsMax parts
+  float4 raw[PF ? kPartsMax : 1][2];
+  auto request = [&](int t) {
+    const float* src = p.logits_in + (((size_t)t * p.L + l) * p.S + s) * E + e0;
+#pragma unroll
+    for (int q = 0; q < kPartsMax; ++q)
+#pragma unroll
+      for (int h = 0; h < 2; ++h)
+        if (q < p.n_partials && e0 + 4 * h < E) raw[q][h] = ldz4<COHERENT>((const float4*)(src + (size_t)q * p.partial_stride + 4 * h));
+  };
+  if (prefetch) request(0);
+
+  for (int t = 0; t < p.n_steps; ++t) {
+    const size_t row = ((size_t)t * p.L + l) * p.S + s;
+
+    // ---- logits of this token: the K parts of the router GEMM summed in a fixed order ---------------------
+    if (!wait(t)) break;
+    float z[kNE];
+    {
+      const float* src = p.logits_in + row * E + e0;
+      if (prefetch) {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (e0 + 4 * h < E) {
+            v = raw[0][h];
+#pragma unroll
+            for (int q = 1; q < kPartsMax; ++q)
+              if (q < p.n_partials) {
+                const float4 u = raw[q][h];
+                v.x = __fadd_rn(v.x, u.x), v.y = __fadd_rn(v.y, u.y), v.z = __fadd_rn(v.z, u.z), v.w = __fadd_rn(v.w, u.w);
+              }
+          }
+          z[4 * h] = v.x, z[4 * h + 1] = v.y, z[4 * h + 2] = v.z, z[4 * h + 3] = v.w;
+        }
+        if (t + 1 < p.n_steps) request(t + 1);
+      } else if (vec4) {
+#pragma unroll
+        for (int i = 0; i < kNE; i += 4) {
+          float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (e0 + i < E) {
+            v = ldz4<COHERENT>((const float4*)(src + i));
+            for (int q = 1; q < p.n_partials; ++q) {
+              const float4 u = ldz4<COHERENT>((const float4*)(src + (size_t)q * p.partial_stride + i));
+              v.x = __fadd_rn(v.x, u.x), v.y = __fadd_rn(v.y, u.y), v.z = __fadd_rn(v.z, u.z), v.w = __fadd_rn(v.w, u.w);
+            }
+          }
+          z[i] = v.x, z[i + 1] = v.y, z[i + 2] = v.z, z[i + 3] = v.w;
+        }
+      } else {
+#pragma unroll
+        for (int i = 0; i < kNE; ++i) {
+          float v = 0.f;
+          if (e0 + i < E) {
+            v = ldz1<COHERENT>(src + i);
+            for (int q = 1; q < p.n_partials; ++q) v = __fadd_rn(v, ldz1<COHERENT>(src + (size_t)q * p.partial_stride + i));
+          }
+          z[i] = v;
+        }
+      }
+      if (p.logits_out != nullptr && active) {
+        float* dst = p.logits_out + row * E + e0;
+        if (vec4) {
+#pragma unroll
+          for (int i = 0; i < kNE; i += 4)
+            if (e0 + i < E) *(float4*)(dst + i) = make_float4(z[i], z[i + 1], z[i + 2], z[i + 3]);
+        } else {
+#pragma unroll
+          for (int i = 0; i < kNE; ++i)
+            if (e0 + i < E) dst[i] = z[i];
+        }
+      }
+    }
+
+    // ---- Eq. 8: range of this token's logits, running mean that includes it ---------------------------------
+    uint32_t kz[kNE];
+    uint32_t kmax_l = 0u, kmin_l = 0xffffffffu;
+#pragma unroll
+    for (int i = 0; i < kNE; ++i) {
+      const bool valid = e0 + i < E;
+      kz[i] = valid ? okey(z[i]) : 0u;
+      kmax_l = max(kmax_l, kz[i]);
+      kmin_l = min(kmin_l, valid ? kz[i] : 0xffffffffu);
+    }
+    const float zmax = okey_inv(group_max<G>(kmax_l));
+    const float zmin = okey_inv(group_min<G>(kmin_l));
+    float delta;
+    if (p.delta_mode == MCCE_DELTA_RUNNING) {
+      sum_range = __fadd_rn(sum_range, __fsub_rn(zmax, zmin));
+      delta = __fdiv_rn(sum_range, (float)(p.cnt0 + (uint32_t)t + 1u));
+    } else {
+      delta = __ldg(p.fixed_delta + l);
+    }
+    const float bias = __fmul_rn(p.lambda, delta);
+
+    // ---- m~_t = cache OR top-J of the router; Eq. 7 -----------------------------------------------------------
+    uint32_t mt = resb;
+    {
+      uint32_t taken = 0u;
+      for (int r = 0; r < p.J; ++r) {
+        const Cand c = group_argmax<G>(kz, kz, taken, e0);
+        if ((c.e >> 3) == sub) taken |= 1u << (c.e & 7);
+      }
+      mt |= taken;
+    }
+    uint32_t kp[kNE];
+#pragma unroll
+    for (int i = 0; i < kNE; ++i) {
+      const float zp = ((mt >> i) & 1u) ? __fadd_rn(z[i], bias) : z[i];
+      kp[i] = e0 + i < E ? okey(zp) : 0u;
+    }
+
+    // ---- top-K of z' in rank order; every lane of the group keeps all K (expert, unmodified logit) pairs --------
+    int sel_e[KMAX];
+    uint32_t sel_k[KMAX];
+    uint32_t miss_bits = 0u, cold_bits = 0u;
+    {
+      uint32_t taken = 0u;
+#pragma unroll
+      for (int r = 0; r < KMAX; ++r) {
+        sel_e[r] = 0, sel_k[r] = 0u;
+        if (r < K) {
+          const Cand c = group_argmax<G>(kp, kz, taken, e0);
+          sel_e[r] = c.e, sel_k[r] = c.z;
+          if ((c.e >> 3) == sub) {
+            const uint32_t bit = 1u << (c.e & 7);
+            taken |= bit;
+            // Eq. 4 against the cache before this token (the owner lane knows)
+            if (!(resb & bit)) miss_bits |= 1u << r;
+            if (!(everb & bit)) cold_bits |= 1u << r;
+          }
+        }
+      }
+    }
+    {
+      const uint32_t both = group_or<G>(miss_bits | (cold_bits << 16));
+      miss_bits = both & 0xffffu, cold_bits = both >> 16;
+    }
+    miss_c += __popc(miss_bits);
+    cold_c += __popc(cold_bits);
+    if (p.miss_trace != nullptr && t < p.trace_avail && sub == 0 && active)
+      p.miss_trace[((size_t)t * p.L + l) * p.S + s] = miss_bits;
+
+    // ---- weights: softmax of the unmodified logits ---------------------------------------------------------------
+    float pe[KMAX], denom = 0.f;
+#pragma unroll
+    for (int r = 0; r < KMAX; ++r) {
+      pe[r] = r < K ? expf(okey_inv(sel_k[r]) - zmax) : 0.f;
+      denom += pe[r];
+    }
+    if (!p.renorm) {
+      float loc = 0.f;
+#pragma unroll
+      for (int i = 0; i < kNE; ++i)
+        if (e0 + i < E) loc += expf(z[i] - zmax);
+      denom = group_sum<G>(loc);
+    }
+
+    // ---- LRU touch: inside the token the higher router weight is the older one -----------------------------------
+    const uint32_t base = (uint32_t)E + (p.tok0 + (uint32_t)t) * (uint32_t)K + 1u;
+#pragma unroll
+    for (int r = 0; r < KMAX; ++r)
+      if (r < K) {
+        int pos = 0;
+#pragma unroll
+        for (int q = 0; q < KMAX; ++q)
+          if (q < K && (sel_k[q] > sel_k[r] || (sel_k[q] == sel_k[r] && sel_e[q] < sel_e[r]))) ++pos;
+        if ((sel_e[r] >> 3) == sub) {
+          const int slot = sel_e[r] & 7;
+#pragma unroll
+          for (int i = 0; i < kNE; ++i)
+            if (i == slot) st[i] = base + (uint32_t)pos;
+          resb |= 1u << slot;
+          everb |= 1u << slot;
+        }
+      }
+    resident += __popc(miss_bits);
+    // evict the resident expert with the smallest recency key until the cache fits (keys of resident experts
+    // are distinct); groups that already fit idle through the loop of their warp's other groups
+    while (__any_sync(kFull, resident > p.C)) {
+      uint32_t lmin = 0xffffffffu;
+#pragma unroll
+      for (int i = 0; i < kNE; ++i)
+        if ((resb >> i) & 1u) lmin = min(lmin, st[i]);
+      const uint32_t m = group_min<G>(lmin);
+      if (resident > p.C) {
+#pragma unroll
+        for (int i = 0; i < kNE; ++i)
+          if (((resb >> i) & 1u) && st[i] == m) st[i] = 0u, resb &= ~(1u << i);
+        --resident;
+      }
+    }
+
+    // ---- results -------------------------------------------------------------------------------------------------------
+    if (sub == 0 && active) {
+      int32_t* so = p.sel_idx + row * K;
+      float* wo = p.sel_w + row * K;
+      if ((K & 3) == 0) {
+#pragma unroll
+        for (int r = 0; r < KMAX; r += 4)
+          if (r < K) {
+            *(int4*)(so + r) = make_int4(sel_e[r], sel_e[r + 1], sel_e[r + 2], sel_e[r + 3]);
+            *(float4*)(wo + r) = make_float4(pe[r] / denom, pe[r + 1] / denom, pe[r + 2] / denom, pe[r + 3] / denom);
+          }
+      } else {
+#pragma unroll
+        for (int r = 0; r < KMAX; ++r)
+          if (r < K) so[r] = sel_e[r], wo[r] = pe[r] / denom;
+      }
+    }
+  }
+
+  // ---- state back to memory ----------------------------------------------------------------------------------------------
+  // ever-resident words: four lanes (32 experts) make one word
+  uint32_t word = everb << (e0 & 31);
+  if (G >= 2) word |= __shfl_xor_sync(kFull, word, 1);
+  if (G >= 4) word |= __shfl_xor_sync(kFull, word, 2);
+  if (active) {
+#pragma unroll
+    for (int i = 0; i < kNE; ++i)
+      if (e0 + i < E) p.stamp[pair * E + e0 + i] = st[i];
+    const int EW = (E + 31) >> 5;
+    if ((sub & 3) == 0 && e0 < E) p.ever[pair * EW + (e0 >> 5)] = word;
+    if (sub == 0) {
+      p.sum_range[pair] = sum_range;
+      p.miss[pair] = miss_c;
+      p.cold[pair] = cold_c;
+    }
+  }
+}
+
+}  // namespace rgroup
+}  // namespace mcce
