@@ -323,6 +323,7 @@ def main_arm(args):
         route_ms = (prof["route"][0] + prof["route_gemm"][0]) / K
         kernels["route"]["achieved_gbs_with_gemm"] = bytes_route / (route_ms * 1e-3) / 1e9
         kernels["route"]["algorithmic_bytes"] = bytes_route
+        kernels["route"]["frac_of_hbm_peak"] = kernels["route"]["achieved_gbs_with_gemm"] / peak
         # grouping + gather: selections in, offsets / permutation out, hidden rows copied into expert order
         bytes_group = wl.L * wl.S * wl.K * (4 + 8) + 2 * wl.L * wl.S * wl.K * wl.d * esz
         kernels["gather"]["achieved_gbs_with_group"] = bytes_group / (
@@ -356,10 +357,12 @@ def main_arm(args):
             eng.route_step(hidden=hidden[:8], n_steps=8, out=(sel8, sw8))
         pr = eng.profile_read(reset=True)
         eng.profile(False)
-        us = 1e3 * (pr["route"][0] / pr["route"][1] + pr["route_gemm"][0] / pr["route_gemm"][1])
+        # with several tokens per launch the GEMM and the tail run as one kernel (no separate GEMM launches)
+        us = 1e3 * (pr["route"][0] + pr["route_gemm"][0]) / max(1, pr["route"][1])
         state_bytes = 2 * (wl.E * 4 + EW * 4 + 12)
         b8 = 8 * (wl.L * wl.S * (wl.d * esz + wl.K * 8) + wl.L * wl.E * wl.d * 4) + wl.L * wl.S * state_bytes
         line["kernels"]["route"]["batched_8_tokens"] = {"us_per_launch": us, "achieved_gbs": b8 / (us * 1e-6) / 1e9,
+                                                        "frac_of_hbm_peak": b8 / (us * 1e-6) / 1e9 / measured_hbm_peak()[0],
                                                         "algorithmic_bytes": b8}
 
     if args.lifetimes:

@@ -11,7 +11,7 @@ CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libmcce.so")
-SOURCES = ["api.cu", "route.cu", "route_thread.cu", "route_static.cu", "route_gemm.cu", "route_gemm_res.cu", "belady.cu", "group.cu", "ffn_simt.cu", "ffn_tc.cu", "gen.cu"]
+SOURCES = ["api.cu", "route.cu", "route_thread.cu", "route_static.cu", "route_gemm.cu", "route_gemm_res.cu", "route_fused.cu", "belady.cu", "group.cu", "ffn_simt.cu", "ffn_tc.cu", "gen.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC,-Wall", "-I", INCLUDE, "-I", CSRC]
 

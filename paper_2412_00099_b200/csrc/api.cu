@@ -50,6 +50,7 @@ struct mcce_ctx {
   RouterGemmPlan rg;
   void* wr_terms;
   float* z_buf;
+  uint32_t* z_ready;
   // optional per-kernel timing: event pairs recorded around each launch, summed by mcce_profile_read
   int profiling;
   int n_pairs;
@@ -88,7 +89,7 @@ bool valid(const mcce_config* c) {
 
 struct Layout {
   size_t stamp, ever, sum_range, miss, cold, err, stats, offsets, perm, inv, Xg, H, O, st_hidden, st_sel, st_w, st_y, st_hidden2, st_sel2, st_w2, st_y2,
-      wr_terms, z_buf, load_tok, life, total;
+      wr_terms, z_buf, z_ready, load_tok, life, total;
 };
 
 Layout layout_of(const mcce_config& c) {
@@ -130,6 +131,7 @@ Layout layout_of(const mcce_config& c) {
   // logits of up to router_gemm_steps_max() tokens; the router-resident kernel writes one array per K part
   const size_t z_slots = (size_t)router_gemm_steps_max() * (router_gemm_res_applicable(c) ? router_gemm_res_parts_max() : 1);
   o.z_buf = take(rg ? z_slots * L * S * E * 4 : 0);
+  o.z_ready = take(rg ? (size_t)router_gemm_steps_max() * L * ((S + 127) / 128) * 4 : 0);   // counters of the fused kernel
   o.load_tok = take(c.track_lifetime ? L * S * E * 4 : 0);
   o.life = take(c.track_lifetime ? L * S * 3 * 8 : 0);
   o.total = p;
@@ -225,7 +227,7 @@ extern "C" int mcce_create(const mcce_config* cfg, void* workspace, size_t works
   ctx->stage_w2 = (float*)(w + lo.st_w2), ctx->stage_y2 = (float*)(w + lo.st_y2);
   ctx->use_tc = cfg->ffn_impl != MCCE_FFN_SIMT && tc_applicable(*cfg);
   ctx->use_tc_router = router_gemm_applicable(*cfg);
-  ctx->wr_terms = w + lo.wr_terms, ctx->z_buf = (float*)(w + lo.z_buf);
+  ctx->wr_terms = w + lo.wr_terms, ctx->z_buf = (float*)(w + lo.z_buf), ctx->z_ready = (uint32_t*)(w + lo.z_ready);
   ctx->load_tok = cfg->track_lifetime ? (uint32_t*)(w + lo.load_tok) : nullptr;
   ctx->life = cfg->track_lifetime ? (unsigned long long*)(w + lo.life) : nullptr;
   cudaError_t e = cudaSetDevice(cfg->device);
@@ -275,6 +277,8 @@ extern "C" int mcce_set_router(mcce_ctx* ctx, const float* Wr, const float* fixe
     if (router_gemm_res_applicable(ctx->cfg)) {
       const int rc2 = router_gemm_res_plan(ctx->cfg, ctx->wr_terms, &ctx->rg);
       if (rc2 != MCCE_OK) return rc2;
+      const int rc3 = route_fused_plan(ctx->cfg, &ctx->rg);
+      if (rc3 != MCCE_OK) return rc3;
     }
     CK(cudaDeviceSynchronize());
   }
@@ -373,6 +377,16 @@ extern "C" int mcce_route_step(mcce_ctx* ctx, int32_t n_steps, const void* hidde
       const int nt = n_steps - t0 < router_gemm_steps_max() ? n_steps - t0 : router_gemm_steps_max();
       const char* h = (const char*)hidden + (size_t)t0 * LS * c.d_model * esz;
       int ks = 1;
+      p.tok0 = (uint32_t)(ctx->tok + t0), p.cnt0 = (uint32_t)(ctx->delta_cnt + t0);
+      p.sel_idx = sel_idx + (size_t)t0 * LS * c.top_k, p.sel_w = sel_w + (size_t)t0 * LS * c.top_k;
+      p.logits_out = logits_out ? logits_out + (size_t)t0 * LS * c.n_experts : nullptr;
+      trace_at(t0, nt);
+      // GEMM and tail in one kernel once there are a few tokens to overlap them over (for one or two tokens
+      // the two launches are faster: measured)
+      if (ctx->rg.fused_ready && nt >= 4) {
+        TIMED(MCCE_K_ROUTE, st, route_fused_launch(ctx->rg, c, h, nt, ctx->z_buf, ctx->z_ready, p, ctx->err, st));
+        continue;
+      }
       if (ctx->rg.res_ready) {
         ks = ctx->rg.res_parts;
         TIMED(MCCE_K_ROUTE_GEMM, st, router_gemm_res_launch(ctx->rg, c, h, nt, ctx->z_buf, ctx->err, st));

@@ -80,6 +80,7 @@ struct RouterGemmPlan {
   uint64_t hidden_rows_res;
   int ready;
   int res_ready, res_parts;   // K parts (= partial logit arrays) of the router-resident kernel
+  int fused_ready, fused_parts;   // the same for the kernel that also runs the routing tail (route_fused.cu)
 };
 bool router_gemm_applicable(const mcce_config& c);
 int router_gemm_steps_max();
@@ -92,6 +93,10 @@ int router_gemm_res_parts_max();
 int router_gemm_res_plan(const mcce_config& c, void* terms, RouterGemmPlan* plan);
 cudaError_t router_gemm_res_launch(RouterGemmPlan& plan, const mcce_config& c, const void* hidden, int n_steps,
                                    float* Z, uint32_t* err, cudaStream_t st);
+
+int route_fused_plan(const mcce_config& c, RouterGemmPlan* plan);
+cudaError_t route_fused_launch(RouterGemmPlan& plan, const mcce_config& c, const void* hidden, int n_steps, float* Z,
+                               uint32_t* ready, RouteParams p, uint32_t* err, cudaStream_t st);
 
 cudaError_t launch_wait_timeout_selftest(uint32_t* err, unsigned long long limit_ns, uint32_t* outcome,
                                          cudaStream_t st);

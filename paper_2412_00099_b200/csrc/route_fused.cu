@@ -3,13 +3,13 @@
 // route_group.cuh run side by side in the same CTAs, so that the tail of one (token, stream tile) overlaps the
 // GEMM of the next ones instead of following it in a second launch.
 //
-// A cluster is the KS CTAs of one layer (one K part of the reduction each).  Warps 0-5 of a CTA are the GEMM
+// A layer belongs to KS CTAs (one K part of the reduction each).  Warps 0-5 of a CTA are the GEMM
 // (TMA producer, MMA issuer, four epilogue warps); they store the partial logits of their K part and then
 // count themselves in on a ready counter of the (layer, token, stream tile).  The remaining warps are the
 // tail: the S streams of the layer are dealt out to the KS CTAs, a group of lanes per stream as in
 // route_group.cuh; before a token they wait until all 4*KS epilogue warps of the layer have counted in, then
-// read the KS partial sums (L2-coherent loads) and route.  A tail warp only ever waits for CTAs of its own
-// cluster, which the hardware schedules together; every wait is bounded in time all the same.
+// read the KS partial sums (L2-coherent loads) and route.  The launch is cooperative, so every CTA that a
+// tail warp waits for is resident; every wait is bounded in time all the same.
 //
 // The accumulation is cut into sets of kSetSlabs K-slabs (the tensor core's fp32 accumulate truncates), each
 // set with its own TMEM columns; the epilogue adds the sets in round-to-nearest fp32.
@@ -35,7 +35,7 @@ constexpr int kPartsMaxF = 8;
 struct FusedArgs {
   int L, S, E, Epad, n_steps;
   int KS, slabs, n_tiles, n_stages;
-  int Sc;               // streams of the layer routed by each CTA of the cluster
+  int Sc;               // streams of the layer routed by each of its CTAs
   int tail_warps;
   uint32_t res_bytes;
   float* Z;             // [KS][n_steps, L, S, E] partial logits
@@ -269,8 +269,8 @@ cudaError_t launch_one(const FusedMaps& m, const FusedArgs& a, const RouteParams
   cfg.gridDim = dim3((unsigned)(a.L * a.KS)), cfg.blockDim = dim3((unsigned)threads);
   cfg.dynamicSmemBytes = (size_t)kSmemMax + 1024, cfg.stream = st;
   cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = (unsigned)a.KS, attr[0].val.clusterDim.y = 1, attr[0].val.clusterDim.z = 1;
+  attr[0].id = cudaLaunchAttributeCooperative;   // all CTAs resident at once, or the launch fails
+  attr[0].val.cooperative = 1;
   cfg.attrs = attr, cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, route_fused_kernel<G, KMAX>, m, a, p);
 }
@@ -282,29 +282,22 @@ cudaError_t launch_g(const FusedMaps& m, const FusedArgs& a, const RouteParams& 
   return launch_one<G, 16>(m, a, p, threads, st);
 }
 
-// Number of clusters of `ks` CTAs of this kernel that the device runs at once (0: not launchable).
+// CTAs of this kernel that the device holds at once (0: not launchable).
 template <int G, int KMAX>
-int active_clusters(int ks, int threads) {
+int resident_ctas(int threads) {
   static int cache[64] = {0};
-  int sms = 0;
+  int sms = 0, per_sm = 0;
   if (sm_count_and_smem_optin(route_fused_kernel<G, KMAX>, (size_t)kSmemMax + 1024, cache, &sms) != cudaSuccess) return 0;
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)(ks * 64)), cfg.blockDim = dim3((unsigned)threads);
-  cfg.dynamicSmemBytes = (size_t)kSmemMax + 1024;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = (unsigned)ks, attr[0].val.clusterDim.y = 1, attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr, cfg.numAttrs = 1;
-  int n = 0;
-  if (cudaOccupancyMaxActiveClusters(&n, route_fused_kernel<G, KMAX>, &cfg) != cudaSuccess) {
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, route_fused_kernel<G, KMAX>, threads,
+                                                    (size_t)kSmemMax + 1024) != cudaSuccess) {
     cudaGetLastError();
     return 0;
   }
-  return n;
+  return per_sm * sms;
 }
-int active_clusters_of(int G, int K, int ks, int threads) {
+int resident_ctas_of(int G, int K, int threads) {
   const int kb = K <= 4 ? 4 : K <= 8 ? 8 : 16;
-#define MCCE_AC(g, k) if (G == g && kb == k) return active_clusters<g, k>(ks, threads);
+#define MCCE_AC(g, k) if (G == g && kb == k) return resident_ctas<g, k>(threads);
   MCCE_AC(1, 4) MCCE_AC(1, 8) MCCE_AC(2, 4) MCCE_AC(2, 8) MCCE_AC(2, 16) MCCE_AC(4, 4) MCCE_AC(4, 8) MCCE_AC(4, 16)
   MCCE_AC(8, 4) MCCE_AC(8, 8) MCCE_AC(8, 16)
 #undef MCCE_AC
@@ -320,8 +313,8 @@ uint32_t res_bytes_of(int slabs, int ks, int Epad) {
 
 // Fixes the K-split of the fused kernel for this configuration, or leaves plan->fused_ready at 0 when the two-kernel
 // path has to be used: other selection rules, lifetime tracking, more than 64 experts, more streams per CTA than
-// its tail warps hold, accumulator sets that do not fit TMEM, clusters that the device cannot place, or so few
-// layers that one cluster per layer would leave most SMs idle.
+// its tail warps hold, accumulator sets that do not fit TMEM, or so few layers that KS CTAs per layer would leave
+// most SMs idle.
 int route_fused_plan(const mcce_config& c, RouterGemmPlan* plan) {
   plan->fused_ready = 0;
   if (!plan->res_ready) return MCCE_OK;
@@ -339,9 +332,9 @@ int route_fused_plan(const mcce_config& c, RouterGemmPlan* plan) {
     const int Sc = (c.n_streams + ks - 1) / ks;
     const int tail_warps = (Sc * G + 31) / 32;
     if (tail_warps > kMaxTailWarps) continue;
-    const int act = active_clusters_of(G, c.top_k, ks, 32 * (kGemmWarps + tail_warps));
-    const int ctas = (act < c.n_layers ? act : c.n_layers) * ks;   // CTAs at work in the first wave
-    if (act >= 1 && ctas > best_ctas) best_ctas = ctas, best_ks = ks;
+    const int ctas = c.n_layers * ks;   // all of them have to be resident together
+    if (ctas <= resident_ctas_of(G, c.top_k, 32 * (kGemmWarps + tail_warps)) && ctas > best_ctas)
+      best_ctas = ctas, best_ks = ks;
   }
   if (best_ks == 0 || 2 * best_ctas < sms) return MCCE_OK;
   plan->fused_parts = best_ks;

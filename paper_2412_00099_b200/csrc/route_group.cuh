@@ -95,13 +95,26 @@ __device__ __forceinline__ float4 ldz4(const float4* q) { return COHERENT ? __ld
 template <bool COHERENT>
 __device__ __forceinline__ float ldz1(const float* q) { return COHERENT ? __ldcg(q) : __ldg(q); }
 
+// What a token contributes before the cache is consulted: its logits, their maximum, the promotion bias
+// lambda * Delta_avg (Eq. 7, Eq. 8) and this lane's bits of the router's own top-J.
+struct Pre {
+  float z[kNE];
+  float zmax, bias;
+  uint32_t topj;
+};
+
 // Routes the p.n_steps tokens of stream s_raw of layer l.  All 32 lanes of a warp must call this together
 // (groups past the last stream run on stream 0's data and store nothing).  `sub` is the lane's index in its
-// group.  wait(t) is called by every lane before the logits of token t are read and returns false to give up.
+// group.  wait(t) is called by every lane before the logits of token t are read and returns false to give up
+// (the same answer in all lanes of a warp).
+//
+// A token's work has a part that does not depend on the cache (logits, range statistic, bias, top-J: stage A)
+// and a part that does (promotion, top-K, misses, LRU: stage B); only B is a chain from token to token.
+// PF: the next token's partial logits are requested while the current token is routed; this assumes that all
+// tokens are there already (a wait() that is always true).
 template <int G, int KMAX, bool PF, bool COHERENT, typename Wait>
 __device__ __forceinline__ void route_group_streams(const RouteParams& p, const int l, const int s_raw, const int sub,
                                                     Wait wait) {
-  // a group past the last stream runs on stream 0's data and stores nothing (its lanes share warps with live groups)
   const bool active = s_raw < p.S;
   const int s = active ? s_raw : 0;
   const size_t pair = (size_t)l * p.S + s;
@@ -112,97 +125,93 @@ __device__ __forceinline__ void route_group_streams(const RouteParams& p, const 
   // ---- state of this (layer, stream) into registers -----------------------------------------------------
   uint32_t st[kNE];
   uint32_t resb = 0u, everb = 0u;   // bit i: this lane's i-th expert is resident / was ever resident
+  int resident = 0;
+  uint32_t miss_c = 0u, cold_c = 0u;
+  float sum_range = 0.f;
   {
     const int EW = (E + 31) >> 5;
     const uint32_t word = e0 < E ? p.ever[pair * EW + (e0 >> 5)] : 0u;
     everb = (word >> (e0 & 31)) & 0xffu;
-  }
 #pragma unroll
-  for (int i = 0; i < kNE; ++i) {
-    st[i] = e0 + i < E ? p.stamp[pair * E + e0 + i] : 0u;
-    resb |= (st[i] != 0u ? 1u : 0u) << i;
+    for (int i = 0; i < kNE; ++i) {
+      st[i] = e0 + i < E ? p.stamp[pair * E + e0 + i] : 0u;
+      resb |= (st[i] != 0u ? 1u : 0u) << i;
+    }
+    resident = (int)group_sum<G>((float)__popc(resb));   // exact: at most 64
+    miss_c = p.miss[pair], cold_c = p.cold[pair];
   }
-  int resident = (int)group_sum<G>((float)__popc(resb));   // exact: at most 64
-  float sum_range = p.sum_range[pair];
-  uint32_t miss_c = p.miss[pair], cold_c = p.cold[pair];
+  sum_range = p.sum_range[pair];
 
   // The partial logits of the next token are requested before the current token is routed, so that their
   // latency (L2, mostly) is off the critical path: up to kPartsMax parts of eight logits per lane in flight.
-  const bool prefetch = PF;   // the launcher checks: rows 16-byte aligned, at most kPartsMax parts
   float4 raw[PF ? kPartsMax : 1][2];
   auto request = [&](int t) {
     const float* src = p.logits_in + (((size_t)t * p.L + l) * p.S + s) * E + e0;
 #pragma unroll
-    for (int q = 0; q < kPartsMax; ++q)
+    for (int q = 0; q < (PF ? kPartsMax : 1); ++q)
 #pragma unroll
       for (int h = 0; h < 2; ++h)
         if (q < p.n_partials && e0 + 4 * h < E) raw[q][h] = ldz4<COHERENT>((const float4*)(src + (size_t)q * p.partial_stride + 4 * h));
   };
-  if (prefetch) request(0);
 
-  for (int t = 0; t < p.n_steps; ++t) {
+  // ---- stage A: logits of token t (the K parts of the router GEMM summed in a fixed order), Eq. 8, top-J -------
+  auto stage_a = [&](const int t, Pre& o) {
     const size_t row = ((size_t)t * p.L + l) * p.S + s;
-
-    // ---- logits of this token: the K parts of the router GEMM summed in a fixed order ---------------------
-    if (!wait(t)) break;
-    float z[kNE];
-    {
-      const float* src = p.logits_in + row * E + e0;
-      if (prefetch) {
+    float (&z)[kNE] = o.z;
+    const float* src = p.logits_in + row * E + e0;
+    if (PF) {
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-          if (e0 + 4 * h < E) {
-            v = raw[0][h];
+      for (int h = 0; h < 2; ++h) {
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (e0 + 4 * h < E) {
+          v = raw[0][h];
 #pragma unroll
-            for (int q = 1; q < kPartsMax; ++q)
-              if (q < p.n_partials) {
-                const float4 u = raw[q][h];
-                v.x = __fadd_rn(v.x, u.x), v.y = __fadd_rn(v.y, u.y), v.z = __fadd_rn(v.z, u.z), v.w = __fadd_rn(v.w, u.w);
-              }
-          }
-          z[4 * h] = v.x, z[4 * h + 1] = v.y, z[4 * h + 2] = v.z, z[4 * h + 3] = v.w;
-        }
-        if (t + 1 < p.n_steps) request(t + 1);
-      } else if (vec4) {
-#pragma unroll
-        for (int i = 0; i < kNE; i += 4) {
-          float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-          if (e0 + i < E) {
-            v = ldz4<COHERENT>((const float4*)(src + i));
-            for (int q = 1; q < p.n_partials; ++q) {
-              const float4 u = ldz4<COHERENT>((const float4*)(src + (size_t)q * p.partial_stride + i));
+          for (int q = 1; q < (PF ? kPartsMax : 1); ++q)
+            if (q < p.n_partials) {
+              const float4 u = raw[q][h];
               v.x = __fadd_rn(v.x, u.x), v.y = __fadd_rn(v.y, u.y), v.z = __fadd_rn(v.z, u.z), v.w = __fadd_rn(v.w, u.w);
             }
-          }
-          z[i] = v.x, z[i + 1] = v.y, z[i + 2] = v.z, z[i + 3] = v.w;
         }
-      } else {
-#pragma unroll
-        for (int i = 0; i < kNE; ++i) {
-          float v = 0.f;
-          if (e0 + i < E) {
-            v = ldz1<COHERENT>(src + i);
-            for (int q = 1; q < p.n_partials; ++q) v = __fadd_rn(v, ldz1<COHERENT>(src + (size_t)q * p.partial_stride + i));
-          }
-          z[i] = v;
-        }
+        z[4 * h] = v.x, z[4 * h + 1] = v.y, z[4 * h + 2] = v.z, z[4 * h + 3] = v.w;
       }
-      if (p.logits_out != nullptr && active) {
-        float* dst = p.logits_out + row * E + e0;
-        if (vec4) {
+      if (t + 1 < p.n_steps) request(t + 1);
+    } else if (vec4) {
 #pragma unroll
-          for (int i = 0; i < kNE; i += 4)
-            if (e0 + i < E) *(float4*)(dst + i) = make_float4(z[i], z[i + 1], z[i + 2], z[i + 3]);
-        } else {
-#pragma unroll
-          for (int i = 0; i < kNE; ++i)
-            if (e0 + i < E) dst[i] = z[i];
+      for (int i = 0; i < kNE; i += 4) {
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (e0 + i < E) {
+          v = ldz4<COHERENT>((const float4*)(src + i));
+          for (int q = 1; q < p.n_partials; ++q) {
+            const float4 u = ldz4<COHERENT>((const float4*)(src + (size_t)q * p.partial_stride + i));
+            v.x = __fadd_rn(v.x, u.x), v.y = __fadd_rn(v.y, u.y), v.z = __fadd_rn(v.z, u.z), v.w = __fadd_rn(v.w, u.w);
+          }
         }
+        z[i] = v.x, z[i + 1] = v.y, z[i + 2] = v.z, z[i + 3] = v.w;
+      }
+    } else {
+#pragma unroll
+      for (int i = 0; i < kNE; ++i) {
+        float v = 0.f;
+        if (e0 + i < E) {
+          v = ldz1<COHERENT>(src + i);
+          for (int q = 1; q < p.n_partials; ++q) v = __fadd_rn(v, ldz1<COHERENT>(src + (size_t)q * p.partial_stride + i));
+        }
+        z[i] = v;
       }
     }
-
-    // ---- Eq. 8: range of this token's logits, running mean that includes it ---------------------------------
+    if (p.logits_out != nullptr && active) {
+      float* dst = p.logits_out + row * E + e0;
+      if (vec4) {
+#pragma unroll
+        for (int i = 0; i < kNE; i += 4)
+          if (e0 + i < E) *(float4*)(dst + i) = make_float4(z[i], z[i + 1], z[i + 2], z[i + 3]);
+      } else {
+#pragma unroll
+        for (int i = 0; i < kNE; ++i)
+          if (e0 + i < E) dst[i] = z[i];
+      }
+    }
+    // Eq. 8: range of this token's logits, running mean that includes it
     uint32_t kz[kNE];
     uint32_t kmax_l = 0u, kmin_l = 0xffffffffu;
 #pragma unroll
@@ -212,35 +221,42 @@ __device__ __forceinline__ void route_group_streams(const RouteParams& p, const 
       kmax_l = max(kmax_l, kz[i]);
       kmin_l = min(kmin_l, valid ? kz[i] : 0xffffffffu);
     }
-    const float zmax = okey_inv(group_max<G>(kmax_l));
+    o.zmax = okey_inv(group_max<G>(kmax_l));
     const float zmin = okey_inv(group_min<G>(kmin_l));
     float delta;
     if (p.delta_mode == MCCE_DELTA_RUNNING) {
-      sum_range = __fadd_rn(sum_range, __fsub_rn(zmax, zmin));
+      sum_range = __fadd_rn(sum_range, __fsub_rn(o.zmax, zmin));
       delta = __fdiv_rn(sum_range, (float)(p.cnt0 + (uint32_t)t + 1u));
     } else {
       delta = __ldg(p.fixed_delta + l);
     }
-    const float bias = __fmul_rn(p.lambda, delta);
-
-    // ---- m~_t = cache OR top-J of the router; Eq. 7 -----------------------------------------------------------
-    uint32_t mt = resb;
-    {
-      uint32_t taken = 0u;
-      for (int r = 0; r < p.J; ++r) {
-        const Cand c = group_argmax<G>(kz, kz, taken, e0);
-        if ((c.e >> 3) == sub) taken |= 1u << (c.e & 7);
-      }
-      mt |= taken;
+    o.bias = __fmul_rn(p.lambda, delta);
+    // this lane's bits of the router's own top-J
+    uint32_t taken = 0u;
+    for (int r = 0; r < p.J; ++r) {
+      const Cand c = group_argmax<G>(kz, kz, taken, e0);
+      if ((c.e >> 3) == sub) taken |= 1u << (c.e & 7);
     }
-    uint32_t kp[kNE];
+    o.topj = taken;
+  };
+
+  // ---- stage B: Eq. 7, top-K, weights, Eq. 4, LRU ---------------------------------------------------------------------
+  auto stage_b = [&](const int t, const Pre& in) {
+    const size_t row = ((size_t)t * p.L + l) * p.S + s;
+    const float (&z)[kNE] = in.z;
+    const float zmax = in.zmax, bias = in.bias;
+    // m~_t = cache OR top-J of the router; z' = z + bias on m~_t
+    const uint32_t mt = resb | in.topj;
+    uint32_t kz[kNE], kp[kNE];
 #pragma unroll
     for (int i = 0; i < kNE; ++i) {
+      const bool valid = e0 + i < E;
       const float zp = ((mt >> i) & 1u) ? __fadd_rn(z[i], bias) : z[i];
-      kp[i] = e0 + i < E ? okey(zp) : 0u;
+      kz[i] = valid ? okey(z[i]) : 0u;
+      kp[i] = valid ? okey(zp) : 0u;
     }
 
-    // ---- top-K of z' in rank order; every lane of the group keeps all K (expert, unmodified logit) pairs --------
+    // top-K of z' in rank order; every lane of the group keeps all K (expert, unmodified logit) pairs
     int sel_e[KMAX];
     uint32_t sel_k[KMAX];
     uint32_t miss_bits = 0u, cold_bits = 0u;
@@ -271,7 +287,7 @@ __device__ __forceinline__ void route_group_streams(const RouteParams& p, const 
     if (p.miss_trace != nullptr && t < p.trace_avail && sub == 0 && active)
       p.miss_trace[((size_t)t * p.L + l) * p.S + s] = miss_bits;
 
-    // ---- weights: softmax of the unmodified logits ---------------------------------------------------------------
+    // weights: softmax of the unmodified logits
     float pe[KMAX], denom = 0.f;
 #pragma unroll
     for (int r = 0; r < KMAX; ++r) {
@@ -286,7 +302,7 @@ __device__ __forceinline__ void route_group_streams(const RouteParams& p, const 
       denom = group_sum<G>(loc);
     }
 
-    // ---- LRU touch: inside the token the higher router weight is the older one -----------------------------------
+    // LRU touch: inside the token the higher router weight is the older one
     const uint32_t base = (uint32_t)E + (p.tok0 + (uint32_t)t) * (uint32_t)K + 1u;
 #pragma unroll
     for (int r = 0; r < KMAX; ++r)
@@ -321,7 +337,7 @@ __device__ __forceinline__ void route_group_streams(const RouteParams& p, const 
       }
     }
 
-    // ---- results -------------------------------------------------------------------------------------------------------
+    // results
     if (sub == 0 && active) {
       int32_t* so = p.sel_idx + row * K;
       float* wo = p.sel_w + row * K;
@@ -338,25 +354,35 @@ __device__ __forceinline__ void route_group_streams(const RouteParams& p, const 
           if (r < K) so[r] = sel_e[r], wo[r] = pe[r] / denom;
       }
     }
+  };
+
+  if (PF) request(0);
+  for (int t = 0; t < p.n_steps; ++t) {
+    if (!wait(t)) break;
+    Pre pre;
+    stage_a(t, pre);
+    stage_b(t, pre);
   }
 
   // ---- state back to memory ----------------------------------------------------------------------------------------------
-  // ever-resident words: four lanes (32 experts) make one word
-  uint32_t word = everb << (e0 & 31);
-  if (G >= 2) word |= __shfl_xor_sync(kFull, word, 1);
-  if (G >= 4) word |= __shfl_xor_sync(kFull, word, 2);
-  if (active) {
+  {
+    // ever-resident words: four lanes (32 experts) make one word
+    uint32_t word = everb << (e0 & 31);
+    if (G >= 2) word |= __shfl_xor_sync(kFull, word, 1);
+    if (G >= 4) word |= __shfl_xor_sync(kFull, word, 2);
+    if (active) {
 #pragma unroll
-    for (int i = 0; i < kNE; ++i)
-      if (e0 + i < E) p.stamp[pair * E + e0 + i] = st[i];
-    const int EW = (E + 31) >> 5;
-    if ((sub & 3) == 0 && e0 < E) p.ever[pair * EW + (e0 >> 5)] = word;
-    if (sub == 0) {
-      p.sum_range[pair] = sum_range;
-      p.miss[pair] = miss_c;
-      p.cold[pair] = cold_c;
+      for (int i = 0; i < kNE; ++i)
+        if (e0 + i < E) p.stamp[pair * E + e0 + i] = st[i];
+      const int EW = (E + 31) >> 5;
+      if ((sub & 3) == 0 && e0 < E) p.ever[pair * EW + (e0 >> 5)] = word;
+      if (sub == 0) {
+        p.miss[pair] = miss_c;
+        p.cold[pair] = cold_c;
+      }
     }
   }
+  if (active && sub == 0) p.sum_range[pair] = sum_range;
 }
 
 }  // namespace rgroup
