@@ -281,6 +281,16 @@ int mcce_selftest_wait_timeout(mcce_ctx* ctx, uint64_t limit_ns);
 /* 1 if mcce_moe_forward of this context runs the tcgen05/TMA expert kernels, 0 if the fp32-pipe ones. */
 int mcce_uses_tensor_path(const mcce_ctx* ctx);
 
+/* Which kernels mcce_route_step runs for a launch of n_tokens tokens from hidden states, once the router is
+ * set (Eq. 3 and the routing rule of Sec. 3.3 either way; this is introspection for tests and benchmarks):
+ * MCCE_ROUTER_FP32_PIPE      the fused route kernel forms the logits itself on the fp32 pipe (fp32 hidden states);
+ * MCCE_ROUTER_GEMM_TAIL      tcgen05 GEMM with the experts as MMA rows, then the routing tail;
+ * MCCE_ROUTER_RESIDENT_TAIL  tcgen05 GEMM with the router resident in shared memory, then the routing tail;
+ * MCCE_ROUTER_FUSED          the router-resident GEMM and the tail in one cooperative kernel.
+ * Negative: an error code. */
+enum { MCCE_ROUTER_FP32_PIPE = 0, MCCE_ROUTER_GEMM_TAIL = 1, MCCE_ROUTER_RESIDENT_TAIL = 2, MCCE_ROUTER_FUSED = 3 };
+int mcce_router_kernel_kind(const mcce_ctx* ctx, int32_t n_tokens);
+
 const char* mcce_strerror(int code);
 int mcce_last_cuda_error(const mcce_ctx* ctx); /* cudaError_t of the last failed CUDA call */
 

@@ -19,11 +19,12 @@ F32, BF16 = 0, 1
 DELTA_RUNNING, DELTA_FIXED = 0, 1
 FFN_AUTO, FFN_SIMT, FFN_TENSOR = 0, 1, 2
 RERANK_CACHE_PRIOR, RERANK_MAX_RANK, RERANK_CUMSUM = 0, 1, 2
+ROUTER_FP32_PIPE, ROUTER_GEMM_TAIL, ROUTER_RESIDENT_TAIL, ROUTER_FUSED = 0, 1, 2, 3
 
 EXPORTS = [
     "mcce_workspace_bytes", "mcce_create", "mcce_destroy", "mcce_set_router", "mcce_set_experts", "mcce_reset",
     "mcce_route_step", "mcce_moe_forward", "mcce_decode_step_host", "mcce_decode_step_chained", "mcce_pipeline_submit_host", "mcce_pipeline_wait", "mcce_cache_stats", "mcce_get_cache_state",
-    "mcce_get_grouping", "mcce_lifetime_stats", "mcce_set_miss_trace", "mcce_belady_replay", "mcce_profile", "mcce_profile_read", "mcce_uses_tensor_path", "mcce_selftest_wait_timeout", "mcce_route_trace_static",
+    "mcce_get_grouping", "mcce_lifetime_stats", "mcce_set_miss_trace", "mcce_belady_replay", "mcce_profile", "mcce_profile_read", "mcce_uses_tensor_path", "mcce_router_kernel_kind", "mcce_selftest_wait_timeout", "mcce_route_trace_static",
     "mcce_route_trace_static_limit", "mcce_gen_normal", "mcce_gen_hidden_step", "mcce_gen_philox_words", "mcce_strerror",
     "mcce_last_cuda_error",
 ]
@@ -80,6 +81,7 @@ def load():
         lib.mcce_set_miss_trace.argtypes = [vp, vp, C.c_int64]
         lib.mcce_belady_replay.argtypes = [vp, i32, i32, i32, i32, i32, vp, i32, vp, vp, vp]
         lib.mcce_uses_tensor_path.argtypes = [vp]
+        lib.mcce_router_kernel_kind.argtypes = [vp, i32]
         lib.mcce_selftest_wait_timeout.argtypes = [vp, C.c_uint64]
         lib.mcce_route_trace_static_limit.restype = C.c_size_t
         lib.mcce_route_trace_static.argtypes = [C.POINTER(Config), i32, vp, vp, vp, vp, vp, vp, C.POINTER(Stats), vp]
@@ -249,6 +251,13 @@ class Engine:
 
     def uses_tensor_path(self) -> bool:
         return self.lib.mcce_uses_tensor_path(self.ctx) == 1
+
+    def router_kernel_kind(self, n_tokens: int = 1) -> int:
+        """ROUTER_FP32_PIPE / ROUTER_GEMM_TAIL / ROUTER_RESIDENT_TAIL / ROUTER_FUSED for a launch of n_tokens."""
+        kind = self.lib.mcce_router_kernel_kind(self.ctx, n_tokens)
+        if kind < 0:
+            _check(kind, self.ctx)
+        return kind
 
     def profile(self, enable: bool):
         _check(self.lib.mcce_profile(self.ctx, int(enable)), self.ctx)

@@ -12,6 +12,9 @@
 using namespace mcce;
 
 constexpr int kMaxPairs = 1024;
+// Tokens of one launch from which mcce_route_step takes the single fused kernel (for fewer the two launches
+// are faster: measured).
+constexpr int kFusedMinTokens = 4;
 
 struct mcce_ctx {
   mcce_config cfg;
@@ -381,9 +384,8 @@ extern "C" int mcce_route_step(mcce_ctx* ctx, int32_t n_steps, const void* hidde
       p.sel_idx = sel_idx + (size_t)t0 * LS * c.top_k, p.sel_w = sel_w + (size_t)t0 * LS * c.top_k;
       p.logits_out = logits_out ? logits_out + (size_t)t0 * LS * c.n_experts : nullptr;
       trace_at(t0, nt);
-      // GEMM and tail in one kernel once there are a few tokens to overlap them over (for one or two tokens
-      // the two launches are faster: measured)
-      if (ctx->rg.fused_ready && nt >= 4) {
+      // GEMM and tail in one kernel once there are a few tokens to overlap them over
+      if (ctx->rg.fused_ready && nt >= kFusedMinTokens) {
         TIMED(MCCE_K_ROUTE, st, route_fused_launch(ctx->rg, c, h, nt, ctx->z_buf, ctx->z_ready, p, ctx->err, st));
         continue;
       }
@@ -707,6 +709,15 @@ extern "C" int mcce_selftest_wait_timeout(mcce_ctx* ctx, uint64_t limit_ns) {
 }
 
 extern "C" int mcce_uses_tensor_path(const mcce_ctx* ctx) { return ctx ? ctx->use_tc : MCCE_EINVAL; }
+
+extern "C" int mcce_router_kernel_kind(const mcce_ctx* ctx, int32_t n_tokens) {
+  if (!ctx || n_tokens < 1) return MCCE_EINVAL;
+  if (!ctx->Wr) return MCCE_ESTATE;
+  if (!(ctx->use_tc_router && ctx->rg.ready)) return MCCE_ROUTER_FP32_PIPE;
+  const int nt = n_tokens < router_gemm_steps_max() ? n_tokens : router_gemm_steps_max();
+  if (ctx->rg.fused_ready && nt >= kFusedMinTokens) return MCCE_ROUTER_FUSED;
+  return ctx->rg.res_ready ? MCCE_ROUTER_RESIDENT_TAIL : MCCE_ROUTER_GEMM_TAIL;
+}
 
 extern "C" int mcce_profile(mcce_ctx* ctx, int enable) {
   if (!ctx) return MCCE_EINVAL;
