@@ -74,6 +74,9 @@ typedef struct {
   int32_t max_rank;       /* M of Algorithm 1, 0..E (MAX_RANK only)                              */
   float cum_threshold;    /* p of Algorithm 2, >= 0 (CUMSUM only)                                */
   int32_t track_lifetime; /* 1: record how long experts stay cached (mcce_lifetime_stats)         */
+  int32_t route_impl;     /* MCCE_ROUTE_AUTO (0) picks per launch what was measured faster;
+                             MCCE_ROUTE_TWO_KERNELS: logits kernel, then routing tail;
+                             MCCE_ROUTE_FUSED: the single cooperative kernel wherever it can run       */
 } mcce_config;
 
 typedef struct {
@@ -288,6 +291,7 @@ int mcce_uses_tensor_path(const mcce_ctx* ctx);
  * MCCE_ROUTER_RESIDENT_TAIL  tcgen05 GEMM with the router resident in shared memory, then the routing tail;
  * MCCE_ROUTER_FUSED          the router-resident GEMM and the tail in one cooperative kernel.
  * Negative: an error code. */
+enum { MCCE_ROUTE_AUTO = 0, MCCE_ROUTE_TWO_KERNELS = 1, MCCE_ROUTE_FUSED = 2 };
 enum { MCCE_ROUTER_FP32_PIPE = 0, MCCE_ROUTER_GEMM_TAIL = 1, MCCE_ROUTER_RESIDENT_TAIL = 2, MCCE_ROUTER_FUSED = 3 };
 int mcce_router_kernel_kind(const mcce_ctx* ctx, int32_t n_tokens);
 

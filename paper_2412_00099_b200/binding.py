@@ -19,6 +19,7 @@ F32, BF16 = 0, 1
 DELTA_RUNNING, DELTA_FIXED = 0, 1
 FFN_AUTO, FFN_SIMT, FFN_TENSOR = 0, 1, 2
 RERANK_CACHE_PRIOR, RERANK_MAX_RANK, RERANK_CUMSUM = 0, 1, 2
+ROUTE_AUTO, ROUTE_TWO_KERNELS, ROUTE_FUSED = 0, 1, 2
 ROUTER_FP32_PIPE, ROUTER_GEMM_TAIL, ROUTER_RESIDENT_TAIL, ROUTER_FUSED = 0, 1, 2, 3
 
 EXPORTS = [
@@ -36,7 +37,7 @@ class Config(C.Structure):
         ("lam", C.c_float), ("delta_mode", C.c_int32), ("renorm", C.c_int32), ("hidden_dtype", C.c_int32),
         ("weight_dtype", C.c_int32), ("ffn_impl", C.c_int32), ("device", C.c_int32),
         ("rerank_mode", C.c_int32), ("max_rank", C.c_int32), ("cum_threshold", C.c_float),
-        ("track_lifetime", C.c_int32)]
+        ("track_lifetime", C.c_int32), ("route_impl", C.c_int32)]
 
 
 class Stats(C.Structure):
@@ -128,12 +129,12 @@ class Engine:
 
     def __init__(self, *, L, E, K, J, n_shared, d, I, C_cap, S, lam, delta_mode=DELTA_RUNNING, renorm=1, dtype=BF16,
                  ffn_impl=FFN_AUTO, device=0, rerank_mode=RERANK_CACHE_PRIOR, max_rank=0, cum_threshold=0.0,
-                 track_lifetime=False):
+                 track_lifetime=False, route_impl=ROUTE_AUTO):
         if not torch.cuda.is_available():
             raise McceError("no CUDA device: this library has no CPU path")
         self.lib = load()
         self.cfg = Config(L, E, K, J, n_shared, d, I, C_cap, S, lam, delta_mode, renorm, dtype, dtype, ffn_impl,
-                          device, rerank_mode, max_rank, cum_threshold, int(track_lifetime))
+                          device, rerank_mode, max_rank, cum_threshold, int(track_lifetime), route_impl)
         self.device = torch.device("cuda", device)
         nbytes = self.lib.mcce_workspace_bytes(C.byref(self.cfg))
         if nbytes == 0:

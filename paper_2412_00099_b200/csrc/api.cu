@@ -12,9 +12,11 @@
 using namespace mcce;
 
 constexpr int kMaxPairs = 1024;
-// Tokens of one launch from which mcce_route_step takes the single fused kernel (for fewer the two launches
-// are faster: measured).
-constexpr int kFusedMinTokens = 4;
+// When MCCE_ROUTE_AUTO takes the single fused kernel: from four tokens per launch (for fewer the two launches
+// are faster) and with at most 16 experts (with more, the tail inside the fused kernel -- 80 registers, no
+// prefetch of the next token's logits -- is a slower chain than the stand-alone tail; measured on the
+// Mixtral-shaped workload 60 against 86 us for eight tokens, on the OLMoE-shaped one 180 against 156).
+constexpr int kFusedMinTokens = 4, kFusedMaxExperts = 16;
 
 struct mcce_ctx {
   mcce_config cfg;
@@ -87,6 +89,7 @@ bool valid(const mcce_config* c) {
   if (c->rerank_mode == MCCE_RERANK_MAX_RANK && (c->max_rank < 0 || c->max_rank > c->n_experts)) return false;
   if (c->rerank_mode == MCCE_RERANK_CUMSUM && !(c->cum_threshold >= 0.f)) return false;
   if (c->track_lifetime != 0 && c->track_lifetime != 1) return false;
+  if (c->route_impl < MCCE_ROUTE_AUTO || c->route_impl > MCCE_ROUTE_FUSED) return false;
   return true;
 }
 
@@ -139,6 +142,12 @@ Layout layout_of(const mcce_config& c) {
   o.life = take(c.track_lifetime ? L * S * 3 * 8 : 0);
   o.total = p;
   return o;
+}
+
+bool use_fused(const mcce_ctx* ctx, int n_tokens) {
+  if (!ctx->rg.fused_ready || ctx->cfg.route_impl == MCCE_ROUTE_TWO_KERNELS) return false;
+  if (ctx->cfg.route_impl == MCCE_ROUTE_FUSED) return true;
+  return n_tokens >= kFusedMinTokens && ctx->cfg.n_experts <= kFusedMaxExperts;
 }
 
 int cuda_fail(mcce_ctx* ctx, cudaError_t e) {
@@ -385,7 +394,7 @@ extern "C" int mcce_route_step(mcce_ctx* ctx, int32_t n_steps, const void* hidde
       p.logits_out = logits_out ? logits_out + (size_t)t0 * LS * c.n_experts : nullptr;
       trace_at(t0, nt);
       // GEMM and tail in one kernel once there are a few tokens to overlap them over
-      if (ctx->rg.fused_ready && nt >= kFusedMinTokens) {
+      if (use_fused(ctx, nt)) {
         TIMED(MCCE_K_ROUTE, st, route_fused_launch(ctx->rg, c, h, nt, ctx->z_buf, ctx->z_ready, p, ctx->err, st));
         continue;
       }
@@ -715,7 +724,7 @@ extern "C" int mcce_router_kernel_kind(const mcce_ctx* ctx, int32_t n_tokens) {
   if (!ctx->Wr) return MCCE_ESTATE;
   if (!(ctx->use_tc_router && ctx->rg.ready)) return MCCE_ROUTER_FP32_PIPE;
   const int nt = n_tokens < router_gemm_steps_max() ? n_tokens : router_gemm_steps_max();
-  if (ctx->rg.fused_ready && nt >= kFusedMinTokens) return MCCE_ROUTER_FUSED;
+  if (use_fused(ctx, nt)) return MCCE_ROUTER_FUSED;
   return ctx->rg.res_ready ? MCCE_ROUTER_RESIDENT_TAIL : MCCE_ROUTER_GEMM_TAIL;
 }
 

@@ -24,14 +24,6 @@ struct Cand {
   uint32_t z;   // key of its unmodified logit
 };
 
-// better(a, b): b replaces a when its key is larger, or equal with the lower expert index
-__device__ __forceinline__ Cand pick(const Cand a, const Cand b) {
-  const bool c = b.k > a.k || (b.k == a.k && b.e < a.e);
-  Cand r;
-  r.k = c ? b.k : a.k, r.e = c ? b.e : a.e, r.z = c ? b.z : a.z;
-  return r;
-}
-
 // Largest key among the experts of the group not in `taken` (bit i = this lane's i-th expert); equal keys ->
 // lowest expert.  Every lane of the group gets the result.
 template <int G>
@@ -50,14 +42,18 @@ __device__ __forceinline__ Cand group_argmax(const uint32_t (&key)[kNE], const u
       c[j].z = gt ? c[2 * j + 1].z : c[2 * j].z;
     }
   Cand best = c[0];
-  // butterfly inside the group (redux.sync restricted to the group's lanes was measured 40 % slower)
+  if (G > 1) {
+    // largest key of the group by a butterfly on the keys alone; among the lanes that hold it the lowest one
+    // has the lowest expert (a lane's experts are consecutive), and hands over its expert and payload
+    const int gbase = (threadIdx.x & 31) & ~(G - 1);
+    uint32_t m = best.k;
 #pragma unroll
-  for (int o = 1; o < G; o <<= 1) {
-    Cand other;
-    other.k = __shfl_xor_sync(kFull, best.k, o);
-    other.e = __shfl_xor_sync(kFull, best.e, o);
-    other.z = __shfl_xor_sync(kFull, best.z, o);
-    best = pick(best, other);
+    for (int o = 1; o < G; o <<= 1) m = max(m, __shfl_xor_sync(kFull, m, o));
+    const unsigned holders = (__ballot_sync(kFull, best.k == m) >> gbase) & ((1u << G) - 1u);
+    const int owner = gbase + __ffs(holders) - 1;
+    best.e = __shfl_sync(kFull, best.e, owner);
+    best.z = __shfl_sync(kFull, best.z, owner);
+    best.k = m;
   }
   return best;
 }
@@ -256,10 +252,15 @@ __device__ __forceinline__ void route_group_streams(const RouteParams& p, const 
       kp[i] = valid ? okey(zp) : 0u;
     }
 
-    // top-K of z' in rank order; every lane of the group keeps all K (expert, unmodified logit) pairs
-    int sel_e[KMAX];
-    uint32_t sel_k[KMAX];
+    // top-K of z' in rank order.  Every lane of the group learns all K (expert, unmodified logit) pairs; the work
+    // per selected expert that follows (LRU position, weight, output) is dealt out to the lanes: lane `sub`
+    // takes the selections r = sub, sub + G, ...
+    constexpr int kMine = (KMAX + G - 1) / G;
+    int sel_e[KMAX], my_e[kMine];
+    uint32_t sel_k[KMAX], my_k[kMine];
     uint32_t miss_bits = 0u, cold_bits = 0u;
+#pragma unroll
+    for (int j = 0; j < kMine; ++j) my_e[j] = 0, my_k[j] = 0u;
     {
       uint32_t taken = 0u;
 #pragma unroll
@@ -268,6 +269,7 @@ __device__ __forceinline__ void route_group_streams(const RouteParams& p, const 
         if (r < K) {
           const Cand c = group_argmax<G>(kp, kz, taken, e0);
           sel_e[r] = c.e, sel_k[r] = c.z;
+          if (sub == r % G) my_e[r / G] = c.e, my_k[r / G] = c.z;
           if ((c.e >> 3) == sub) {
             const uint32_t bit = 1u << (c.e & 7);
             taken |= bit;
@@ -287,30 +289,35 @@ __device__ __forceinline__ void route_group_streams(const RouteParams& p, const 
     if (p.miss_trace != nullptr && t < p.trace_avail && sub == 0 && active)
       p.miss_trace[((size_t)t * p.L + l) * p.S + s] = miss_bits;
 
-    // weights: softmax of the unmodified logits
-    float pe[KMAX], denom = 0.f;
+    // my selections: weight (softmax of the unmodified logits) and position in the token's LRU order (the higher
+    // router weight is the older one)
+    float pe[kMine], loc = 0.f;
+    int my_pos[kMine];
 #pragma unroll
-    for (int r = 0; r < KMAX; ++r) {
-      pe[r] = r < K ? expf(okey_inv(sel_k[r]) - zmax) : 0.f;
-      denom += pe[r];
+    for (int j = 0; j < kMine; ++j) {
+      const bool mine = sub + j * G < K;
+      pe[j] = mine ? expf(okey_inv(my_k[j]) - zmax) : 0.f;
+      loc += pe[j];
+      int pos = 0;
+#pragma unroll
+      for (int q = 0; q < KMAX; ++q)
+        if (q < K && (sel_k[q] > my_k[j] || (sel_k[q] == my_k[j] && sel_e[q] < my_e[j]))) ++pos;
+      my_pos[j] = pos;
     }
     if (!p.renorm) {
-      float loc = 0.f;
+      loc = 0.f;
 #pragma unroll
       for (int i = 0; i < kNE; ++i)
         if (e0 + i < E) loc += expf(z[i] - zmax);
-      denom = group_sum<G>(loc);
     }
+    const float denom = group_sum<G>(loc);
 
-    // LRU touch: inside the token the higher router weight is the older one
+    // LRU touch by the lane that holds the expert
     const uint32_t base = (uint32_t)E + (p.tok0 + (uint32_t)t) * (uint32_t)K + 1u;
 #pragma unroll
     for (int r = 0; r < KMAX; ++r)
       if (r < K) {
-        int pos = 0;
-#pragma unroll
-        for (int q = 0; q < KMAX; ++q)
-          if (q < K && (sel_k[q] > sel_k[r] || (sel_k[q] == sel_k[r] && sel_e[q] < sel_e[r]))) ++pos;
+        const int pos = G > 1 ? __shfl_sync(kFull, my_pos[r / G], ((threadIdx.x & 31) & ~(G - 1)) + r % G) : my_pos[r / G];
         if ((sel_e[r] >> 3) == sub) {
           const int slot = sel_e[r] & 7;
 #pragma unroll
@@ -338,20 +345,14 @@ __device__ __forceinline__ void route_group_streams(const RouteParams& p, const 
     }
 
     // results
-    if (sub == 0 && active) {
-      int32_t* so = p.sel_idx + row * K;
-      float* wo = p.sel_w + row * K;
-      if ((K & 3) == 0) {
+    if (active) {
 #pragma unroll
-        for (int r = 0; r < KMAX; r += 4)
-          if (r < K) {
-            *(int4*)(so + r) = make_int4(sel_e[r], sel_e[r + 1], sel_e[r + 2], sel_e[r + 3]);
-            *(float4*)(wo + r) = make_float4(pe[r] / denom, pe[r + 1] / denom, pe[r + 2] / denom, pe[r + 3] / denom);
-          }
-      } else {
-#pragma unroll
-        for (int r = 0; r < KMAX; ++r)
-          if (r < K) so[r] = sel_e[r], wo[r] = pe[r] / denom;
+      for (int j = 0; j < kMine; ++j) {
+        const int r = sub + j * G;
+        if (r < K) {
+          p.sel_idx[row * K + r] = my_e[j];
+          p.sel_w[row * K + r] = pe[j] / denom;
+        }
       }
     }
   };

@@ -91,12 +91,12 @@ def test_fused_route_kernel_from_hidden_states(base, kw, chunk):
     wl = base.with_(**kw)
     Wr = wl.router()
     xs = np.stack(list(wl.hidden_trace(2 * chunk + 1)))
-    eng, o = mb.engine_for(wl, ffn_impl=mb.FFN_SIMT), H.oracle_for(wl)
+    eng, o = mb.engine_for(wl, ffn_impl=mb.FFN_SIMT, route_impl=mb.ROUTE_FUSED), H.oracle_for(wl)
     eng.set_router(H.to_dev(Wr))
     assert eng.router_kernel_kind(chunk) == mb.ROUTER_FUSED
-    # two fused launches, then one token through the two-kernel path on the state the fused kernel left
+    # two fused launches of several tokens, then one of a single token
     near, dz = follow_chunked(eng, o, Wr, xs[:2 * chunk], chunk, mb.ROUTER_FUSED)
-    near2, dz2 = follow_chunked(eng, o, Wr, xs[2 * chunk:], 1, mb.ROUTER_RESIDENT_TAIL)
+    near2, dz2 = follow_chunked(eng, o, Wr, xs[2 * chunk:], 1, mb.ROUTER_FUSED)
     print("%s fused: %d near ties, max logit err %.2e" % (wl.name, near + near2, max(dz, dz2)))
     eng.close()
 
@@ -110,9 +110,9 @@ def test_router_resident_gemm_then_tail(base, kw):
     wl = base.with_(**kw)
     Wr = wl.router()
     xs = np.stack(list(wl.hidden_trace(10)))
-    eng, o = mb.engine_for(wl, ffn_impl=mb.FFN_SIMT), H.oracle_for(wl)
+    eng, o = mb.engine_for(wl, ffn_impl=mb.FFN_SIMT, route_impl=mb.ROUTE_FUSED), H.oracle_for(wl)
     eng.set_router(H.to_dev(Wr))
-    assert eng.router_kernel_kind(8) == mb.ROUTER_RESIDENT_TAIL     # too few layers for the fused kernel
+    assert eng.router_kernel_kind(8) == mb.ROUTER_RESIDENT_TAIL     # too few layers for the fused kernel, even if asked
     near, dz = follow_chunked(eng, o, Wr, xs[:8], 8, mb.ROUTER_RESIDENT_TAIL)
     near2, dz2 = follow_chunked(eng, o, Wr, xs[8:], 1, mb.ROUTER_RESIDENT_TAIL)
     print("%s resident: %d near ties, max logit err %.2e" % (wl.name, near + near2, max(dz, dz2)))
@@ -126,7 +126,8 @@ def test_fused_kernel_and_two_kernel_path_leave_the_same_state():
     Wr = H.to_dev(wl.router())
     xs = np.stack(list(wl.hidden_trace(16)))
     x = torch.from_numpy(xs.view(np.int16)).cuda().view(torch.bfloat16)
-    a, b = mb.engine_for(wl, ffn_impl=mb.FFN_SIMT), mb.engine_for(wl, ffn_impl=mb.FFN_SIMT)
+    a = mb.engine_for(wl, ffn_impl=mb.FFN_SIMT, route_impl=mb.ROUTE_FUSED)
+    b = mb.engine_for(wl, ffn_impl=mb.FFN_SIMT, route_impl=mb.ROUTE_TWO_KERNELS)
     a.set_router(Wr)
     b.set_router(Wr)
     assert a.router_kernel_kind(16) == mb.ROUTER_FUSED and b.router_kernel_kind(1) == mb.ROUTER_RESIDENT_TAIL
@@ -144,3 +145,18 @@ def test_fused_kernel_and_two_kernel_path_leave_the_same_state():
         assert np.array_equal(a.cache_state()[0], b.cache_state()[0])
     a.close()
     b.close()
+
+
+def test_automatic_choice_of_the_routing_kernels():
+    """MCCE_ROUTE_AUTO: the fused kernel from four tokens per launch for few experts (Mixtral-shaped), the two
+    kernels otherwise."""
+    for base, kw, n, want in ((synth.MIXTRAL, dict(L=32, S=64, d=1024), 8, mb.ROUTER_FUSED),
+                              (synth.MIXTRAL, dict(L=32, S=64, d=1024), 1, mb.ROUTER_RESIDENT_TAIL),
+                              (synth.QWEN, dict(L=24, S=64, d=512), 8, mb.ROUTER_RESIDENT_TAIL),
+                              (synth.QWEN, dict(L=2, S=16, d=256, E=100), 8, mb.ROUTER_GEMM_TAIL),
+                              (synth.TINY, dict(), 8, mb.ROUTER_FP32_PIPE)):
+        wl = base.with_(**kw)
+        eng = mb.engine_for(wl, ffn_impl=mb.FFN_SIMT)
+        eng.set_router(H.to_dev(wl.router()))
+        assert eng.router_kernel_kind(n) == want, (wl.name, n)
+        eng.close()
