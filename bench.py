@@ -33,7 +33,7 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel (ffn_up), per layer,
 # from the ncu capture summarised in profiles/step_kernels_qwen_4layers.md (a 4-layer case; traffic
 # grows in proportion to the layer count).  Workloads without a capture of the current kernel: None.
-NCU_TRAFFIC_BYTES_PER_LAYER = {"qwen1.5-moe-a2.7b-shaped": (2976824000 + 25219328) / 4}
+NCU_TRAFFIC_BYTES_PER_LAYER = {"qwen1.5-moe-a2.7b-shaped": (2977804000 + 26244608) / 4}
 
 
 def parse_args():
@@ -54,6 +54,11 @@ def parse_args():
     ap.add_argument("--chained", action="store_true",
                     help="sequential-layer mode: the layers of a token chained through a residual stream (L rounds "
                          "of single-layer launches per step) instead of independent layers")
+    ap.add_argument("--route-only", action="store_true",
+                    help="routing alone (router logits, promotion, top-K, miss counting, LRU): no expert weights, "
+                         "--route-tokens tokens per launch; one step = one launch")
+    ap.add_argument("--route-tokens", type=int, default=8, help="tokens per launch with --route-only")
+    ap.add_argument("--route-impl", default="auto", choices=["auto", "two", "fused"])
     ap.add_argument("--impl", default="mcce", choices=["mcce", "reference"])
     ap.add_argument("--ffn", default="auto", choices=["auto", "simt", "tensor"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -197,6 +202,81 @@ def measured_hbm_peak():
         except (KeyError, ValueError):
             pass
     return FALLBACK_HBM_GBS, "fallback (earlier pool measurement)"
+
+
+def route_only_arm(args):
+    """Routing alone on one GPU: hidden states resident in HBM, --route-tokens tokens per launch."""
+    import torch
+
+    from paper_2412_00099_b200 import binding as mb
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    dev = torch.device("cuda", 0)
+    wl = workload_of(args)
+    n, W, K = args.route_tokens, args.warmup, args.steps
+    impl = {"auto": mb.ROUTE_AUTO, "two": mb.ROUTE_TWO_KERNELS, "fused": mb.ROUTE_FUSED}[args.route_impl]
+    # the expert buffers of the context are not used: smallest intermediate size, no shared experts
+    eng = mb.engine_for(wl, n_shared=0, I=8, ffn_impl=mb.FFN_SIMT, route_impl=impl)
+    wdt = torch.bfloat16 if wl.bf16 else torch.float32
+    Wr = mb.gen_normal(torch.empty((wl.L, wl.E, wl.d), dtype=torch.float32, device=dev), wl.seed, synth.T_ROUTER,
+                       std=wl.weight_std)
+    eng.set_router(Wr)
+    slots = 6                                                   # launches cycle over 6 * n tokens of hidden states
+    hidden = torch.empty((slots * n, wl.L, wl.S, wl.d), dtype=wdt, device=dev)
+    state = torch.empty(wl.L * wl.S * wl.d, dtype=torch.float32, device=dev)
+    for t in range(slots * n):
+        mb.gen_hidden_step(state, hidden[t], wl.seed, t, wl.rho, wl.topic_offset)
+    sel = torch.empty((n, wl.L, wl.S, wl.K), dtype=torch.int32, device=dev)
+    sw = torch.empty((n, wl.L, wl.S, wl.K), dtype=torch.float32, device=dev)
+
+    def step(i):
+        o = (i % slots) * n
+        eng.route_step(hidden=hidden[o:o + n], n_steps=n, out=(sel, sw))
+
+    for i in range(W):
+        step(i)
+    eng.profile(True)
+    eng.profile_read(reset=True)
+    torch.cuda.synchronize(dev)
+    props = torch.cuda.get_device_properties(dev)
+    sampler = ClockSampler("GPU-" + str(props.uuid)) if hasattr(props, "uuid") else None
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(W, W + K):
+        step(i)
+    e1.record()
+    torch.cuda.synchronize(dev)
+    ms_total = e0.elapsed_time(e1)
+    clocks = sampler.stop() if sampler else {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+    prof = eng.profile_read(reset=True)
+    eng.profile(False)
+    total, _ = eng.cache_stats()
+    esz = 2 if wl.bf16 else 4
+    EW = (wl.E + 31) // 32
+    # per launch: hidden rows and results of n tokens, the router once per token, cache state in and out once
+    alg = n * (wl.L * wl.S * (wl.d * esz + wl.K * 8) + wl.L * wl.E * wl.d * 4) + wl.L * wl.S * 2 * (wl.E * 4 + EW * 4 + 12)
+    launches = prof["route"][1] + prof["route_gemm"][1]
+    kern_ms = (prof["route"][0] + prof["route_gemm"][0]) / K
+    peak, peak_src = measured_hbm_peak()
+    achieved = alg / (kern_ms * 1e-3) / 1e9
+    kind = {mb.ROUTER_FP32_PIPE: "fp32-pipe logits inside the route kernel", mb.ROUTER_GEMM_TAIL: "tcgen05 GEMM, then tail",
+            mb.ROUTER_RESIDENT_TAIL: "router-resident tcgen05 GEMM, then tail",
+            mb.ROUTER_FUSED: "router-resident tcgen05 GEMM and tail in one cooperative kernel"}[eng.router_kernel_kind(n)]
+    line = {"metric": METRIC + ", routing only", "value": wl.S * wl.L * n * K / (ms_total * 1e-3), "unit": UNIT, "n_gpus": 1,
+            "steps": K, "warmup": W, "ms_per_step": ms_total / K, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16" if wl.bf16 else "f32", "data": "synthetic",
+            "config": config_of(wl, {"route_only": True, "tokens_per_launch": n, "kernels": kind,
+                                     "l2": "hidden states of %d launches cycled (%.0f MB, larger than L2)"
+                                           % (slots, slots * n * wl.L * wl.S * wl.d * esz / 1e6)}),
+            "miss_rate": total[2] / max(1, total[1]),
+            "roofline": {"kernel": "routing step (logits + tail)", "bound": "hbm", "achieved": achieved, "peak": peak,
+                         "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src, "traffic": None,
+                         "algorithmic_bytes_per_launch": alg, "avg_launch_ms": kern_ms},
+            "kernels": {k: {"ms_per_step": v[0] / K, "launches": v[1]} for k, v in prof.items() if v[1]},
+            "gpu_launches": launches, "clocks": clocks}
+    print(json.dumps(line), flush=True)
+    eng.close()
 
 
 def main_arm(args):
@@ -419,5 +499,7 @@ if __name__ == "__main__":
     a = parse_args()
     if a.impl == "reference":
         reference_arm(a)
+    elif a.route_only:
+        route_only_arm(a)
     else:
         main_arm(a)
