@@ -395,8 +395,16 @@ extern "C" int mcce_route_step(mcce_ctx* ctx, int32_t n_steps, const void* hidde
       trace_at(t0, nt);
       // GEMM and tail in one kernel once there are a few tokens to overlap them over
       if (use_fused(ctx, nt)) {
-        TIMED(MCCE_K_ROUTE, st, route_fused_launch(ctx->rg, c, h, nt, ctx->z_buf, ctx->z_ready, p, ctx->err, st));
-        continue;
+        cudaError_t fe = cudaSuccess;
+        const int rc_f = timed(ctx, MCCE_K_ROUTE, st, [&]() {
+          fe = route_fused_launch(ctx->rg, c, h, nt, ctx->z_buf, ctx->z_ready, p, ctx->err, st);
+          return fe == cudaErrorCooperativeLaunchTooLarge ? cudaSuccess : fe;
+        });
+        if (rc_f != MCCE_OK) return rc_f;
+        if (fe == cudaSuccess) continue;
+        // the device cannot hold the whole grid at once (it is shared with other work): two kernels from now on
+        cudaGetLastError();
+        ctx->rg.fused_ready = 0;
       }
       if (ctx->rg.res_ready) {
         ks = ctx->rg.res_parts;
