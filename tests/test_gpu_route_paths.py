@@ -14,7 +14,18 @@ from tests.test_gpu_parity import ROUTE_CASES, ar1_logits
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("E,K,J,C,lam,dm,renorm,quant", [c for c in ROUTE_CASES if c[0] <= 64])
+GROUP_CASES = [c for c in ROUTE_CASES if c[0] <= 64] + [
+    # E,  K, J, C,  lam, delta_mode, renorm, quant
+    (64, 16, 3, 40, 0.5, 0, 1, None),      # two selections per lane of an eight-lane group
+    (64, 12, 2, 10, 0.8, 0, 0, 0.25),      # C < K, K not a multiple of 4, no renormalisation, ties
+    (16, 16, 2, 8, 0.5, 0, 1, None),       # K = E with two lanes per stream
+    (8, 8, 1, 3, 0.7, 1, 1, 0.5),          # K = E with one lane per stream, fixed Delta
+    (24, 7, 7, 24, 0.3, 0, 1, None),       # four lanes per stream, the last lane empty
+    (57, 9, 0, 57, 1.0, 0, 1, 0.125),      # odd expert count: scalar loads of the logits
+]
+
+
+@pytest.mark.parametrize("E,K,J,C,lam,dm,renorm,quant", GROUP_CASES)
 @pytest.mark.parametrize("chunk", [1, 5])
 def test_group_tail_from_logits_is_bit_exact(E, K, J, C, lam, dm, renorm, quant, chunk):
     """Without lifetime tracking and with at most 64 experts the group-of-lanes tail runs (one to eight lanes
