@@ -87,6 +87,23 @@ static void top_by_value(const float* v, int n, int count, int32_t* out) {
   }
 }
 
+/* Sec. 3.2 (Cumsum-Threshold): the number M of top-ranked experts to consider is the smallest one whose
+   router probabilities add up to at least p; all n if they never do.  w_by_rank[i] is the probability of
+   the expert of rank i.  mass[i] = probability of the first i ranks, added rank by rank in fp32; M is the
+   first i with mass[i] >= p.  *distance (optional) receives how far p lies from the two partial sums on
+   either side of the decision, mass[M] - p and p - mass[M-1], whichever is smaller (infinite when M = 0 or
+   when p is never reached): a step with a tiny distance could resolve either way in another arithmetic. */
+static int ranks_for_mass(const float* w_by_rank, int n, float p, float* distance) {
+  float mass[ORC_MAX_E + 1];
+  mass[0] = 0.0f;
+  for (int i = 0; i < n; ++i) mass[i + 1] = mass[i] + w_by_rank[i];
+  int M = n, reached = 0;
+  for (int i = n; i >= 0; --i)
+    if (mass[i] >= p) M = i, reached = 1;
+  if (distance) *distance = (reached && M > 0) ? fminf(mass[M] - p, p - mass[M - 1]) : INFINITY;
+  return M;
+}
+
 /* ---------------------------------------------------------------------------------------------- */
 /* Eq. 3: z = G(x) = W_r x, accumulated in double, rounded once to fp32.                            */
 /* x_dtype: 0 = fp32, 1 = bf16 stored as uint16.                                                    */
@@ -188,20 +205,12 @@ void orc_route_slab(const orc_config* c, const float* z_all /*[L,S,E]*/,
         for (int e = 0; e < E; ++e) in_cache[e] = stamp[e] != 0;
         int M = c->max_rank;
         if (c->rerank_mode == 2) {
-          /* Algorithm 2: M = smallest count of top-ranked experts whose probabilities reach p. */
+          /* Algorithm 2 / Sec. 3.2: M from the router probabilities (softmax of z) in rank order. */
           double denom = 0.0;
+          float w_by_rank[ORC_MAX_E];
           for (int e = 0; e < E; ++e) denom += exp((double)z[e] - (double)zmax);
-          float p_cum = 0.0f;
-          M = 0;
-          while (p_cum < c->cum_threshold && M < E) {
-            M += 1;
-            const float wr = (float)(exp((double)z[r[M - 1]] - (double)zmax) / denom);
-            const float before = p_cum;
-            p_cum = p_cum + wr;
-            /* distance of the threshold from the two partial sums that decided M */
-            if (p_cum >= c->cum_threshold)
-              cum_margin = fminf(p_cum - c->cum_threshold, c->cum_threshold - before);
-          }
+          for (int i = 0; i < E; ++i) w_by_rank[i] = (float)(exp((double)z[r[i]] - (double)zmax) / denom);
+          M = ranks_for_mass(w_by_rank, E, c->cum_threshold, &cum_margin);
         }
         orc_max_rank(r, E, in_cache, M, J, rank);
       }
@@ -424,16 +433,13 @@ void orc_max_rank(const int32_t* r, int n, const uint8_t* in_cache, int M, int J
   orc_promote(r, J, tmp, n, out);
 }
 
-/* Algorithm 2 (Cumsum-Threshold): M = smallest rank count whose router probabilities sum to >= p,
-   then Max-Rank with that M.  w[e] are the softmax weights; returns the M it used. */
+/* Algorithm 2 / Sec. 3.2 (Cumsum-Threshold): Max-Rank with M = the smallest number of top ranks whose
+   router probabilities sum to at least p.  w[e] are the softmax weights; returns the M it used. */
 int orc_cumsum_threshold(const int32_t* r, int n, const float* w, const uint8_t* in_cache, float p,
                          int J, int32_t* out /*[n]*/) {
-  float p_cum = 0.0f;
-  int M = 0;
-  while (p_cum < p && M < n) {
-    M += 1;
-    p_cum = p_cum + w[r[M - 1]];
-  }
+  float w_by_rank[ORC_MAX_E];
+  for (int i = 0; i < n; ++i) w_by_rank[i] = w[r[i]];
+  const int M = ranks_for_mass(w_by_rank, n, p, NULL);
   orc_max_rank(r, n, in_cache, M, J, out);
   return M;
 }

@@ -46,9 +46,18 @@ MUTATIONS = [
     ("promote keeps the subset in place", "for (int i = 0; i < n_subset; ++i) out[n++] = subset[i];\n  for (int i = 0; i < n_all; ++i) {",
      "for (int i = 0; i < 0; ++i) out[n++] = subset[i];\n  for (int i = 0; i < n_all; ++i) {\n    if (n_subset >= 0) { out[n++] = all[i]; continue; }"),
     ("max-rank window off by one", "for (int i = 0; i < M && i < n; ++i)", "for (int i = 0; i <= M && i < n; ++i)"),
-    ("cumulative threshold strict", "while (p_cum < p && M < n) {", "while (p_cum <= p && M < n) {"),
-    ("cumulative threshold strict in the routing mode", "while (p_cum < c->cum_threshold && M < E) {",
-     "while (p_cum <= c->cum_threshold && M < E) {"),
+    ("cumulative threshold strict", "if (mass[i] >= p) M = i, reached = 1;", "if (mass[i] > p) M = i, reached = 1;"),
+    ("cumulative mass skips the first rank", "mass[i + 1] = mass[i] + w_by_rank[i];",
+     "mass[i + 1] = mass[i] + w_by_rank[i < n - 1 ? i + 1 : i];"),
+    ("near-tie margin ignores the K / K+1 gap of the promoted logits",
+     "if (K < E && c->rerank_mode == 0) m = fminf(m, zp[rank[K - 1]] - zp[rank[K]]);", ";"),
+    ("near-tie margin takes the K / K+1 gap from the unmodified logits",
+     "if (K < E && c->rerank_mode == 0) m = fminf(m, zp[rank[K - 1]] - zp[rank[K]]);",
+     "if (K < E && c->rerank_mode == 0) m = fminf(m, z[rank[K - 1]] - z[rank[K]]);"),
+    ("near-tie margin ignores the top-J boundary", "m = fminf(m, z[tj[J - 1]] - z[tj[J]]);", ";"),
+    ("near-tie margin ignores the in-token order", "for (int r = 0; r + 1 < K; ++r) m = fminf(m, zsel[order[r]] - zsel[order[r + 1]]);", ";"),
+    ("near-tie margin ignores the distance to the cumulative threshold", "m = fminf(m, cum_margin);", ";"),
+    ("threshold distance one-sided", "fminf(mass[M] - p, p - mass[M - 1])", "(mass[M] - p)"),
     ("Belady evicts the nearest next use", "if (next > victim_next) {", "if (victim_next < 0 || next < victim_next) {"),
     ("lifetime counted from the first token", "const int64_t life = tok - load_tok_all[p * E + victim];", "const int64_t life = tok;"),
 ]
@@ -74,7 +83,8 @@ def run_pins():
              (pins.test_max_rank_over_all_ranks_is_the_saturated_cache_prior, (1,)),
              (pins.test_lifetimes_match_brute_force_over_resident_sets, ()),
              (pins.test_cumsum_mode_reaches_the_threshold_exactly, ()),
-             (pins.test_miss_trace_matches_resident_sets, ())]
+             (pins.test_miss_trace_matches_resident_sets, ()),
+             (pins.test_near_tie_margin_hand_instances, ())]
     failed = []
     for fn, args in calls:
         try:

@@ -632,3 +632,37 @@ def test_miss_trace_matches_resident_sets():
             assert int(o.last_miss_mask[0, s]) == want
             total += bin(want).count("1")
     assert total == o.stats()[0][2]
+
+
+def test_near_tie_margin_hand_instances():
+    """The near-tie report (the smallest gap that decided an outcome of the step) on instances worked by hand,
+    one per kind of gap: K-th against (K+1)-th promoted logit (Eq. 7), the top-J boundary of the unmodified
+    logits (Sec. 3.3), neighbours in the in-token eviction order (Sec. 4.2), and the distance of the cumulative
+    probability from the threshold (Algorithm 2).  All values are dyadic, so the expected gaps are exact."""
+    def one(z, E, K, J, C, lam, cached=(), fixed=1.0, mode=0, p=0.0):
+        cfg = orc.OracleConfig(1, E, K, J, 0, 16, 8, C, 1, lam, 1, 1, 0, mode, 0, p)
+        o = orc.Oracle(cfg, fixed_delta=np.array([fixed], np.float32))
+        if cached:
+            init = np.full((1, 1, C), -1, np.int32)
+            init[0, 0, :len(cached)] = cached
+            o.reset(init_order=init)
+        sel, _, margin, _ = o.route(np.array(z, np.float32).reshape(1, 1, E), want_margin=True)
+        return sel[0, 0].tolist(), float(margin[0, 0])
+
+    # (a) expert 3 is cached and gets the bias 1.0: z' = [2, 1.5, 1.25, 1.75]; the second and third largest
+    #     promoted logits are 1.75 and 1.5 -> 0.25 (the selected pair's own logits, 2 and 0.75, lie 1.25 apart)
+    assert one([2.0, 1.5, 1.25, 0.75], 4, 2, 0, 2, 1.0, cached=(3,)) == ([0, 3], 0.25)
+    # (b) J = 1: the router's first and second choice lie 0.0625 apart; expert 2 is cached and promoted by 4 to
+    #     4.5, far from everything else (K boundary 4.5 - 1.9375, in-token order 2.0 - 0.5)
+    assert one([2.0, 1.9375, 0.5, 0.25], 4, 2, 1, 2, 1.0, cached=(2,), fixed=4.0) == ([0, 2], 0.0625)
+    # (c) nothing cached, J = 0: the two selected experts lie 0.03125 apart (which of them is evicted first),
+    #     the K boundary 0.96875
+    assert one([1.0, 0.96875, 0.0, -1.0], 4, 2, 0, 2, 0.5) == ([0, 1], 0.03125)
+    # (d) Algorithm 2: probabilities 4/7, 2/7, 1/7; p = 0.7 is passed by the second rank (6/7), and lies
+    #     0.7 - 4/7 = 0.128571 above the first partial sum; neighbouring logits are ln 2 apart
+    ln2 = float(np.log(2.0))
+    sel, m = one([2 * ln2, ln2, 0.0], 3, 1, 0, 2, 0.5, mode=2, p=0.7)
+    assert sel == [0] and abs(m - (0.7 - 4.0 / 7.0)) < 1e-6
+    # ... and with p = 0.5 the first rank alone passes it, 4/7 - 0.5 = 0.0714 beyond
+    sel, m = one([2 * ln2, ln2, 0.0], 3, 1, 0, 2, 0.5, mode=2, p=0.5)
+    assert abs(m - (4.0 / 7.0 - 0.5)) < 1e-6
