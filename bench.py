@@ -30,10 +30,39 @@ from paper_2412_00099_b200 import synth  # noqa: E402
 METRIC = "cache-aware MoE decode steps/s (stream*token*layer)"
 UNIT = "steps/s"
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel (ffn_up), per layer,
-# from the ncu capture summarised in profiles/step_kernels_qwen_4layers.md (a 4-layer case; traffic
-# grows in proportion to the layer count).  Workloads without a capture of the current kernel: None.
-NCU_TRAFFIC_BYTES_PER_LAYER = {"qwen1.5-moe-a2.7b-shaped": (2977804000 + 26244608) / 4}
+# DRAM counters of the dominant kernel from an ncu capture of a small case, kept as a tracked data file beside
+# its summary; the sources of the kernel are hashed into it, so that a figure taken from an older kernel is
+# not reported for the current one.
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "ffn_up_dram_traffic.json")
+KERNEL_SOURCES = ("paper_2412_00099_b200/csrc/ffn_tc.cu", "paper_2412_00099_b200/csrc/tc_common.cuh")
+
+
+def kernel_sources_sha():
+    import hashlib
+    h = hashlib.sha256()
+    for rel in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, rel), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def measured_traffic(workload_name, n_layers, default_config):
+    """(bytes per launch, source) of ffn_up from the tracked capture: the capture's per-layer DRAM bytes (read +
+    write) times the layers of this run -- the kernel streams every layer's experts once, so its traffic grows in
+    proportion to the layer count.  (None, why) when there is no capture of this workload in its default
+    configuration, or when the kernel's sources have changed since the capture."""
+    try:
+        rec = json.load(open(TRAFFIC_FILE))
+    except (OSError, ValueError):
+        return None, "no capture on file"
+    cap = rec.get("captures", {}).get(workload_name)
+    if cap is None or not default_config:
+        return None, "no capture of this configuration"
+    if rec.get("kernel_sources_sha16") != kernel_sources_sha():
+        return None, "kernel sources changed since the capture in profiles/%s" % os.path.basename(TRAFFIC_FILE)
+    per_layer = (cap["dram_bytes_read"] + cap["dram_bytes_write"]) / cap["layers"]
+    return per_layer * n_layers, "profiles/%s: %s, %d-layer capture scaled by layers (%d / %d)" % (
+        os.path.basename(TRAFFIC_FILE), cap["kernel"], cap["layers"], n_layers, cap["layers"])
 
 
 def parse_args():
@@ -63,6 +92,10 @@ def parse_args():
     ap.add_argument("--ffn", default="auto", choices=["auto", "simt", "tensor"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--step-by-step", action="store_true",
+                    help="one mcce_route_step + mcce_moe_forward per token on one stream instead of mcce_pipeline_submit")
+    ap.add_argument("--no-steady-state", action="store_true",
+                    help="skip the 200-step steady-state region that follows a shorter timed region")
     ap.add_argument("--no-kernel-timing", action="store_true",
                     help="do not bracket each kernel with CUDA events (no roofline block; shows their overhead)")
     return ap.parse_args()
@@ -324,8 +357,14 @@ def main_arm(args):
 
     # ---- hidden-state trace for warm-up + timed steps, resident in HBM ---------------------------------
     W, K = args.warmup, args.steps
-    n_tok = W + K
+    # a steady-state region of STEADY steps follows the timed one when that is shorter (a short region runs
+    # before the GPU has settled at its power cap and reads a few per cent faster)
+    STEADY = 200
+    steady = (not args.no_steady_state) and not args.chained and K < STEADY
+    n_tok = W + K + (STEADY if steady else 0)
     per_tok = wl.L * wl.S * wl.d * (2 if wl.bf16 else 4)
+    if steady and n_tok * per_tok > 12e9:
+        steady, n_tok = False, W + K
     if n_tok * per_tok > 24e9:
         raise SystemExit("hidden trace of %d tokens does not fit the budget; use fewer steps" % n_tok)
     hidden = torch.empty((n_tok, wl.L, wl.S, wl.d), dtype=wdt, device=dev)
@@ -334,14 +373,18 @@ def main_arm(args):
         mb.gen_hidden_step(state, hidden[t], seed, t, wl.rho, wl.topic_offset)
     sel = torch.empty((1, wl.L, wl.S, wl.K), dtype=torch.int32, device=dev)
     sw = torch.empty((1, wl.L, wl.S, wl.K), dtype=torch.float32, device=dev)
-    y = torch.empty((wl.L, wl.S, wl.d), dtype=torch.float32, device=dev)
+    y = torch.empty((2, wl.L, wl.S, wl.d), dtype=torch.float32, device=dev)
+    torch.cuda.synchronize(dev)          # the pipelined entry point reads hidden on a stream of its own
 
     def step(t):
         if args.chained:
             eng.decode_step_chained(hidden[t, 0])
-            return
-        eng.route_step(hidden=hidden[t], out=(sel, sw))
-        eng.moe_forward(hidden[t], sel[0], sw[0], out=y)
+        elif args.step_by_step:
+            eng.route_step(hidden=hidden[t], out=(sel, sw))
+            eng.moe_forward(hidden[t], sel[0], sw[0], out=y[0])
+        else:
+            # routing + grouping of this token on the library's internal stream, overlapping the previous token's experts
+            eng.pipeline_submit(hidden[t], y[t & 1])
 
     def barrier():
         if world > 1:
@@ -357,10 +400,11 @@ def main_arm(args):
     sampler = ClockSampler("GPU-" + str(props.uuid)) if hasattr(props, "uuid") else None
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
-    for t in range(W, n_tok):
+    for t in range(W, W + K):
         step(t)
     e1.record()
     barrier()
+    eng.pipeline_wait()
     ms_total = reduce_max(e0.elapsed_time(e1), dev if world > 1 else None)
     clocks = sampler.stop() if sampler else {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
     prof = eng.profile_read(reset=True)
@@ -368,6 +412,22 @@ def main_arm(args):
 
     units_per_step = wl.S * wl.L                      # per rank
     value = world * units_per_step * K / (ms_total * 1e-3)
+    steady_rec = None
+    if steady:
+        barrier()
+        sampler = ClockSampler("GPU-" + str(props.uuid)) if hasattr(props, "uuid") else None
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s0.record()
+        for t in range(W + K, W + K + STEADY):
+            step(t)
+        s1.record()
+        barrier()
+        eng.pipeline_wait()
+        ms_steady = reduce_max(s0.elapsed_time(s1), dev if world > 1 else None)
+        steady_rec = {"steps": STEADY, "value": world * units_per_step * STEADY / (ms_steady * 1e-3), "unit": UNIT,
+                      "ms_per_step": ms_steady / STEADY,
+                      "clocks": sampler.stop() if sampler else {"sm_mhz": None, "sm_max_mhz": None, "reasons": []},
+                      "note": "the same step for %d more tokens right after the timed region" % STEADY}
     total, _ = eng.cache_stats()
     miss_rate = total[2] / max(1, total[1])
     misses = reduce_sum(total[2], dev if world > 1 else None)
@@ -378,22 +438,32 @@ def main_arm(args):
     touched = int((np.diff(offsets, axis=1) > 0).sum()) + wl.L * wl.n_shared
     rows = wl.L * wl.S * (wl.K + wl.n_shared)
     esz = 2 if wl.bf16 else 4
-    bytes_up = touched * 2 * wl.d * wl.I * esz + rows * wl.d * esz + rows * wl.I * esz
+    bytes_up_weights = touched * 2 * wl.d * wl.I * esz
+    bytes_up = bytes_up_weights + rows * wl.d * esz + rows * wl.I * esz
     # down projection: weights + H rows; the tensor path adds into y (L*S*d fp32) in its epilogue, the
     # fp32-pipe path writes one fp32 row per (pair) for a separate combine pass
     bytes_down = touched * wl.d * wl.I * esz + rows * wl.I * esz + (
         wl.L * wl.S * wl.d * 4 if _uses_tensor(eng) else rows * wl.d * 4)
-    roofline, kernels = None, {}
+    roofline, roofline_route, kernels = None, None, {}
     if not args.no_kernel_timing:
         up_ms, up_n = prof["ffn_up"]
         peak, peak_src = measured_hbm_peak()
-        achieved = bytes_up / (up_ms / max(1, up_n) * 1e-3) / 1e9
+        up_launch_s = up_ms / max(1, up_n) * 1e-3
+        # algorithmic bytes of the gate/up kernel: the gate and up matrices of every touched expert, once
+        achieved = bytes_up_weights / up_launch_s / 1e9
+        default_cfg = args.cache is None and args.layers is None
+        traffic, traffic_src = (measured_traffic(synth.ALIASES[args.workload].name, wl.L, default_cfg)
+                                if _uses_tensor(eng) else (None, "no capture of the fp32-pipe kernels"))
         roofline = {"kernel": "ffn_up (H = silu(X Wg^T) * (X Wu^T), all expert groups)", "bound": "hbm",
                     "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
-                    "traffic": (NCU_TRAFFIC_BYTES_PER_LAYER[synth.ALIASES[args.workload].name] * wl.L
-                                if _uses_tensor(eng) and synth.ALIASES[args.workload].name in NCU_TRAFFIC_BYTES_PER_LAYER
-                                and args.cache is None else None), "algorithmic_bytes_per_launch": bytes_up,
+                    "traffic": traffic, "traffic_source": traffic_src,
+                    "algorithmic_bytes_per_launch": bytes_up_weights,
+                    "algorithmic_bytes_definition": "2 * d * I * 2 B per touched expert (gate and up weights, read once)",
+                    "achieved_with_activation_rows": bytes_up / up_launch_s / 1e9,
                     "avg_launch_ms": up_ms / max(1, up_n)}
+        if achieved > peak:
+            roofline["note"] = ("above 1: the peak is a copy (half reads, half writes); a kernel that almost only "
+                                "reads can exceed it")
         kernels = {k: {"ms_per_step": v[0] / K, "launches": v[1]} for k, v in prof.items()}
         dn_ms, dn_n = prof["ffn_down"]
         kernels["ffn_down"]["achieved_gbs"] = bytes_down / (dn_ms / max(1, dn_n) * 1e-3) / 1e9
@@ -404,6 +474,11 @@ def main_arm(args):
         kernels["route"]["achieved_gbs_with_gemm"] = bytes_route / (route_ms * 1e-3) / 1e9
         kernels["route"]["algorithmic_bytes"] = bytes_route
         kernels["route"]["frac_of_hbm_peak"] = kernels["route"]["achieved_gbs_with_gemm"] / peak
+        roofline_route = {"kernel": "routing step inside the decode step (logits + tail, one token per launch)",
+                          "bound": "hbm", "achieved": kernels["route"]["achieved_gbs_with_gemm"], "peak": peak,
+                          "unit": "GB/s", "frac": kernels["route"]["frac_of_hbm_peak"], "traffic": None,
+                          "algorithmic_bytes_per_launch": bytes_route, "avg_launch_ms": route_ms,
+                          "note": "one token per launch is bound by launch and fill latency, not by HBM"}
         # grouping + gather: selections in, offsets / permutation out, hidden rows copied into expert order
         bytes_group = wl.L * wl.S * wl.K * (4 + 8) + 2 * wl.L * wl.S * wl.K * wl.d * esz
         kernels["gather"]["achieved_gbs_with_group"] = bytes_group / (
@@ -416,14 +491,21 @@ def main_arm(args):
                                            % ((bytes_up + bytes_down) / 1e9),
                                      "ffn_path": "tensor" if _uses_tensor(eng) else "simt",
                                      "layer_mode": "chained through a residual stream" if args.chained else "independent",
+                                     "call": ("mcce_decode_step_chained" if args.chained else
+                                              "mcce_route_step + mcce_moe_forward per token" if args.step_by_step else
+                                              "mcce_pipeline_submit (device buffers)"),
                                      "rerank": args.rerank if args.rerank == "prior" else (
                                          "maxrank M=%d" % max_rank if args.rerank == "maxrank"
                                          else "cumsum p=%g" % args.cum_p),
                                      "experts_touched_per_step": touched}),
-            "miss_rate": misses / max(1, selections), "roofline": roofline, "kernels": kernels,
-            # kernels of this library launched in the timed region (on the tensor path the "combine" slot is
-            # a memset of y, not a kernel, and is not counted)
-            "gpu_launches": K * 6, "clocks": clocks}
+            "miss_rate": misses / max(1, selections), "roofline": roofline, "roofline_route": roofline_route,
+            "kernels": kernels,
+            # kernels of this library launched in the timed region: counted by the library itself (one count per
+            # bracketed launch) when kernel timing is on
+            "gpu_launches": (sum(v[1] for v in prof.values()) if not args.no_kernel_timing else None),
+            "clocks": clocks}
+    if steady_rec:
+        line["steady_state"] = steady_rec
 
     # ---- routing alone, several tokens per launch (state stays in registers, the GEMM sees more tiles) -----
     if not args.no_kernel_timing and wl.bf16 and n_tok >= 8 and not args.chained:
@@ -444,6 +526,8 @@ def main_arm(args):
         line["kernels"]["route"]["batched_8_tokens"] = {"us_per_launch": us, "achieved_gbs": b8 / (us * 1e-6) / 1e9,
                                                         "frac_of_hbm_peak": b8 / (us * 1e-6) / 1e9 / measured_hbm_peak()[0],
                                                         "algorithmic_bytes": b8}
+        if line["roofline_route"] is not None:
+            line["roofline_route"]["eight_tokens_per_launch"] = line["kernels"]["route"]["batched_8_tokens"]
 
     if args.lifetimes:
         (n_ev, mean, sd), _ = eng.lifetimes()

@@ -12,8 +12,8 @@
  * sequential because the cache state carries over.
  *
  * Ownership: the caller owns every buffer, including the workspace, and keeps them alive until
- * mcce_destroy.  The library allocates no device memory and creates no streams (except the two copy
- * streams of mcce_pipeline_submit_host).  Weights are borrowed.
+ * mcce_destroy.  The library allocates no device memory and creates no streams (except the three internal
+ * streams of the pipelined entry points).  Weights are borrowed.
  * Errors: every call returns 0 on success or a negative MCCE_E* code; nothing throws, aborts or prints.
  * Kernel launches are asynchronous on the given stream unless a function says that it synchronises.
  * A context is not thread-safe; distinct contexts are independent.
@@ -35,7 +35,11 @@ enum {
   MCCE_ESTATE = -3,   /* weights not set, or a counter would overflow (reset needed)    */
   MCCE_ECUDA = -4,    /* a CUDA call failed; see mcce_last_cuda_error                   */
   MCCE_ETIMEOUT = -5, /* a bounded wait inside a kernel gave up; the context stays usable */
-  MCCE_ELIMIT = -6    /* problem larger than the fixed array of mcce_route_trace_static   */
+  MCCE_ELIMIT = -6,   /* problem larger than the fixed array of mcce_route_trace_static   */
+  MCCE_EINDEX = -7,   /* an expert id outside [0, E) reached the grouping pass (the pair was skipped), or a
+                         check of the checked mode failed: a grouping position outside [0, S*K), more than C
+                         resident experts, or two resident experts with the same recency key               */
+  MCCE_ENONFINITE = -8 /* checked mode: a router logit was NaN or infinite                               */
 };
 
 enum { MCCE_F32 = 0, MCCE_BF16 = 1 };
@@ -77,6 +81,15 @@ typedef struct {
   int32_t route_impl;     /* MCCE_ROUTE_AUTO (0) picks per launch what was measured faster;
                              MCCE_ROUTE_TWO_KERNELS: logits kernel, then routing tail;
                              MCCE_ROUTE_FUSED: the single cooperative kernel wherever it can run       */
+  int32_t deterministic;  /* 1: y = sum_k w_k E_k(x) + shared experts is added in slot order on every path, so
+                             that repeated runs give identical bits (the paper's runs are deterministic,
+                             Sec. 4.1); the tensor-core path then writes one fp32 row per (stream, slot) and
+                             sums them in a second pass instead of adding into y with atomics              */
+  int32_t checked;        /* 1: checked mode.  Every routing launch is followed by kernels that verify the
+                             logits (finite), the cache state (at most C resident experts per (stream,
+                             layer), distinct recency keys) and every grouping pass (positions inside
+                             [0, S*K)); a violation is recorded and reported by mcce_cache_stats as
+                             MCCE_ENONFINITE / MCCE_EINDEX.  Costs a few small launches per call          */
 } mcce_config;
 
 typedef struct {
@@ -123,6 +136,8 @@ int mcce_reset(mcce_ctx* ctx, const int32_t* init_order, int keep_delta_stats, c
  *   sel_idx    DEVICE int32 [n_steps,L,S,K] out, rank order of z'
  *   sel_w      DEVICE fp32  [n_steps,L,S,K] out
  *   logits_out DEVICE fp32  [n_steps,L,S,E] out, optional: the logits the decision was taken on
+ * When E is a multiple of 4, rows of logits are read and written four floats at a time: logits_in and
+ * logits_out must then be 16-byte aligned (MCCE_EINVAL otherwise; 4-byte alignment suffices for other E).
  */
 int mcce_route_step(mcce_ctx* ctx, int32_t n_steps, const void* hidden, const float* logits_in,
                     int32_t* sel_idx, float* sel_w, float* logits_out, void* cuda_stream);
@@ -133,7 +148,10 @@ int mcce_route_step(mcce_ctx* ctx, int32_t n_steps, const void* hidden, const fl
  *   y DEVICE fp32 [L,S,d] out.
  * With bf16 weights the intermediate silu(g)*u is rounded to bf16 before the down projection.  On the
  * tensor-core path the K + n_shared terms of a stream are added into y with fp32 atomic adds in no fixed
- * order, so the last bits of y may differ between runs (the fp32-pipe path sums in slot order). */
+ * order, so the last bits of y may differ between runs, unless the configuration sets `deterministic`
+ * (the fp32-pipe path always sums in slot order).
+ * An entry of sel_idx outside [0, E) (padding, an uninitialised buffer) is skipped: the pair contributes
+ * nothing to y, and the next mcce_cache_stats reports MCCE_EINDEX. */
 int mcce_moe_forward(mcce_ctx* ctx, const void* hidden, const int32_t* sel_idx, const float* sel_w,
                      float* y, void* cuda_stream);
 
@@ -155,23 +173,42 @@ int mcce_decode_step_chained(mcce_ctx* ctx, const void* x0, void* x_out, int32_t
 int mcce_decode_step_host(mcce_ctx* ctx, const void* hidden_host, float* y_host, int32_t* sel_idx_host,
                           void* cuda_stream);
 
-/* The same decode step, pipelined over successive tokens: copies overlap the compute of neighbouring steps.
- * mcce_pipeline_submit_host enqueues, without waiting, the upload of hidden_host [L,S,d] on an internal
- * copy-in stream, route + experts on cuda_stream once the upload has landed, and the download of y
- * [L,S,d] (and sel_idx [L,S,K] if non-NULL) on an internal copy-out stream once the step has finished.
- * Two staging slots alternate: a call blocks only if the step submitted two calls earlier has not yet left
- * the device, so the upload of token t+1 and the download of token t-1 run while token t computes.  The
- * host buffers of a submitted step must stay valid, and y_host must not be read, until mcce_pipeline_wait
+/* The same decode step, pipelined over successive tokens.  Routing needs only the hidden states of its token and
+ * the cache state that the previous token's routing left (Sec. 3.3: the mask m_t is the cache after token t-1),
+ * not the previous token's experts; so routing, grouping and the row copy of step t+1 run on an internal stream
+ * while the expert kernels of step t, which stream all the weights, still run on cuda_stream.  Two sets of
+ * buffers ("slots") alternate.
+ *
+ * mcce_pipeline_submit_host enqueues, without waiting, the upload of hidden_host [L,S,d] on an internal copy-in
+ * stream, the step, and the download of y [L,S,d] (and sel_idx [L,S,K] if non-NULL) on an internal copy-out
+ * stream once the step has finished.  A call blocks only if the step submitted two calls earlier has not yet
+ * left the device, so the upload of token t+1 and the download of token t-1 also run while token t computes.
+ * The host buffers of a submitted step must stay valid, and y_host must not be read, until mcce_pipeline_wait
  * (or the second following submit) returns.  hidden_host / y_host must be pinned for the copies to be
- * asynchronous.  The two copy streams and their events are the only CUDA objects the library creates (on
- * the first submit); it still allocates no device memory.  Always use the same cuda_stream per context. */
+ * asynchronous.
+ *
+ * mcce_pipeline_submit is its twin for DEVICE buffers: hidden [L,S,d] (hidden_dtype), y [L,S,d] fp32 out, sel_idx
+ * [L,S,K] int32 out or NULL.  Nothing is copied.  The library reads `hidden` on its internal stream, which does
+ * not wait for cuda_stream: hidden must be complete when the call is made, or hidden_ready (a cudaEvent_t, may be
+ * NULL) must mark its completion.  y and sel_idx are complete in cuda_stream order.  y is cleared on the internal
+ * stream while the previous step may still compute: consecutive calls must use different y buffers, and neither
+ * hidden nor y of a step may be touched by the caller until that step has finished on cuda_stream.
+ *
+ * The three internal streams and their events are the only CUDA objects the library creates (on the first
+ * submit); it still allocates no device memory.  Always use the same cuda_stream per context, and call
+ * mcce_pipeline_wait before using any other entry point of the context that routes or runs experts. */
 int mcce_pipeline_submit_host(mcce_ctx* ctx, const void* hidden_host, float* y_host, int32_t* sel_idx_host,
                               void* cuda_stream);
-/* Waits until every submitted step has been copied back. */
+int mcce_pipeline_submit(mcce_ctx* ctx, const void* hidden /*DEVICE*/, float* y /*DEVICE*/, int32_t* sel_idx /*DEVICE*/,
+                         void* hidden_ready /*cudaEvent_t or NULL*/, void* cuda_stream);
+/* Waits until every submitted step has finished (and, for host buffers, has been copied back). */
 int mcce_pipeline_wait(mcce_ctx* ctx);
 
 /* Eq. 4 counters, summed over streams: total and per layer (HOST [L], may be NULL).  Synchronises.
- * Also reports MCCE_ETIMEOUT if any kernel of this context gave up on a bounded wait. */
+ * The counters are always written; the return value also carries what the kernels of this context recorded
+ * since the last mcce_reset, in this order of precedence: MCCE_ETIMEOUT (a bounded wait gave up),
+ * MCCE_EINDEX (an expert id out of range was skipped, or a check of the checked mode failed),
+ * MCCE_ENONFINITE (checked mode: a non-finite logit). */
 int mcce_cache_stats(mcce_ctx* ctx, mcce_stats* total /*HOST*/, mcce_stats* per_layer /*HOST*/);
 
 /* Cache lifetimes (the statistic of the paper's Table 2): a lifetime is the number of tokens from the
@@ -189,6 +226,15 @@ int mcce_lifetime_stats(mcce_ctx* ctx, mcce_lifetime* total /*HOST*/, mcce_lifet
  * are not recorded; recording restarts at entry 0 when the buffer is set and after mcce_reset.  NULL with
  * capacity 0 turns it off. */
 int mcce_set_miss_trace(mcce_ctx* ctx, uint32_t* trace, int64_t capacity_tokens);
+
+/* Logit range from a calibration set (appendix "Logit Range Estimation": Delta_avg estimated once over a
+ * calibration set instead of during inference).  After some tokens have been routed in MCCE_DELTA_RUNNING
+ * mode, writes for every layer the mean over its streams of the running estimate of Eq. 8,
+ *   delta[l] = (1/S) sum_s sum_range[l][s] / tokens,
+ * accumulated in double precision and rounded once to fp32: the constants to hand to mcce_set_router of a
+ * context in MCCE_DELTA_FIXED mode.  delta HOST fp32 [L].  MCCE_ESTATE if no token has been routed yet.
+ * Synchronises. */
+int mcce_calibrate_delta(mcce_ctx* ctx, float* delta /*HOST*/);
 
 /* Canonical cache state: order HOST int32 [L,S,C] most-recently-used first, -1 padded; optional
  * ever HOST uint8 [L,S,E]; delta_sum HOST fp32 [L,S] and *delta_count (optional).  Synchronises. */
@@ -234,8 +280,9 @@ int mcce_gen_philox_words(uint32_t* out, uint64_t start_block, uint64_t n_blocks
  * (HOST arrays of MCCE_N_KERNELS entries), clearing the sums if reset != 0. */
 enum {
   MCCE_K_ROUTE = 0,    /* fused route kernel (with bf16 hidden states: its tail, on the logits of MCCE_K_ROUTE_GEMM) */
-  MCCE_K_GROUP = 1,    /* histogram + scan + scatter                 */
-  MCCE_K_GATHER = 2,   /* activation rows into expert order (clears y on the tensor-core path) */
+  MCCE_K_GROUP = 1,    /* grouping, first pass: histograms of the selected experts per chunk of pairs */
+  MCCE_K_GATHER = 2,   /* grouping, second pass: scan, stable scatter, and the activation rows copied into expert
+                          order on the way (clears y on the tensor-core path) */
   MCCE_K_FFN_UP = 3,   /* H = silu(X Wg^T) * (X Wu^T), all groups    */
   MCCE_K_FFN_DOWN = 4, /* O = H Wd^T, all groups                     */
   MCCE_K_COMBINE = 5,  /* weighted sum over slots + shared experts (fp32-pipe path; fused into FFN_DOWN otherwise) */
@@ -250,14 +297,18 @@ int mcce_profile_read(mcce_ctx* ctx, double* ms /*HOST*/, int64_t* launches /*HO
  * decisions: a server whose memory pool already owns the whole GPU, a plug-in that only receives input
  * and output buffers, or a latency-critical callback that must not enter the allocator.
  *
- * Runs the same fused route kernel as mcce_route_step over n_steps tokens of every (stream, layer),
- * starting from EMPTY caches, zero counters and (running mode) an empty Delta statistic.  The cache
+ * Routes n_steps tokens of every (stream, layer) with the routing kernels of mcce_route_step, starting from
+ * EMPTY caches, zero counters and (running mode) an empty Delta statistic.  From hidden states the logits
+ * are formed on the fp32 pipe for both hidden dtypes (a context given bf16 hidden states uses the tensor
+ * cores instead, so its logits can differ in the last bits and, at a near tie, so can a selection).  The cache
  * state it needs while it runs lives in a fixed array inside the library image
  * (mcce_route_trace_static_limit() bytes = 4 MiB, resident on every GPU that loads the library until
  * the process exits) instead of in a workspace.  The state needs about L*S*(4*E + 4*ceil(E/32) + 12)
  * bytes; a configuration that does not fit is refused with MCCE_ELIMIT and nothing is launched.
- *   cfg         HOST; n_layers, n_streams, n_experts, top_k, top_j, cache_capacity, lambda,
- *               delta_mode, renorm, hidden_dtype and d_model are used, the rest is ignored
+ *   cfg         HOST; n_layers, n_streams, n_experts, top_k, top_j, cache_capacity, lambda, delta_mode,
+ *               renorm, hidden_dtype, d_model, rerank_mode, max_rank and cum_threshold are used and checked
+ *               as in mcce_create; the rest is ignored
+ *               (hidden must be 16-byte aligned, and so must logits_in when E is a multiple of 4)
  *   hidden, Wr  DEVICE [n_steps,L,S,d] (hidden_dtype) and fp32 [L,E,d], or both NULL
  *   logits_in   DEVICE fp32 [n_steps,L,S,E], or NULL; exactly one of hidden / logits_in is given
  *   fixed_delta DEVICE fp32 [L], only for MCCE_DELTA_FIXED
@@ -265,7 +316,8 @@ int mcce_profile_read(mcce_ctx* ctx, double* ms /*HOST*/, int64_t* launches /*HO
  *   totals_host HOST, optional: Eq. 4 counters summed over everything; asking for them makes the call
  *               wait for the stream, otherwise it only enqueues work
  * The device that is current when the call is made is used.  The first call on each device looks up
- * the array's device address; make that first call outside any stream capture.  The call uses no
+ * the array's device address and keeps it for the life of the process; make that first call outside any
+ * stream capture, and do not call again on a device after cudaDeviceReset (the address is then stale).  The call uses no
  * cudaMalloc / cudaFree and no allocating library routine.  Every call on a device shares the one
  * array and first clears the part it uses, so nothing carries over between calls -- and two calls
  * whose GPU work overlaps (different streams, or different host threads) race on it: serialise them. */

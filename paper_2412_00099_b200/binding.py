@@ -24,7 +24,7 @@ ROUTER_FP32_PIPE, ROUTER_GEMM_TAIL, ROUTER_RESIDENT_TAIL, ROUTER_FUSED = 0, 1, 2
 
 EXPORTS = [
     "mcce_workspace_bytes", "mcce_create", "mcce_destroy", "mcce_set_router", "mcce_set_experts", "mcce_reset",
-    "mcce_route_step", "mcce_moe_forward", "mcce_decode_step_host", "mcce_decode_step_chained", "mcce_pipeline_submit_host", "mcce_pipeline_wait", "mcce_cache_stats", "mcce_get_cache_state",
+    "mcce_route_step", "mcce_moe_forward", "mcce_decode_step_host", "mcce_decode_step_chained", "mcce_pipeline_submit_host", "mcce_pipeline_submit", "mcce_pipeline_wait", "mcce_cache_stats", "mcce_calibrate_delta", "mcce_get_cache_state",
     "mcce_get_grouping", "mcce_lifetime_stats", "mcce_set_miss_trace", "mcce_belady_replay", "mcce_profile", "mcce_profile_read", "mcce_uses_tensor_path", "mcce_router_kernel_kind", "mcce_selftest_wait_timeout", "mcce_route_trace_static",
     "mcce_route_trace_static_limit", "mcce_gen_normal", "mcce_gen_hidden_step", "mcce_gen_philox_words", "mcce_strerror",
     "mcce_last_cuda_error",
@@ -37,7 +37,8 @@ class Config(C.Structure):
         ("lam", C.c_float), ("delta_mode", C.c_int32), ("renorm", C.c_int32), ("hidden_dtype", C.c_int32),
         ("weight_dtype", C.c_int32), ("ffn_impl", C.c_int32), ("device", C.c_int32),
         ("rerank_mode", C.c_int32), ("max_rank", C.c_int32), ("cum_threshold", C.c_float),
-        ("track_lifetime", C.c_int32), ("route_impl", C.c_int32)]
+        ("track_lifetime", C.c_int32), ("route_impl", C.c_int32), ("deterministic", C.c_int32),
+        ("checked", C.c_int32)]
 
 
 class Stats(C.Structure):
@@ -74,8 +75,10 @@ def load():
         lib.mcce_decode_step_host.argtypes = [vp] * 5
         lib.mcce_decode_step_chained.argtypes = [vp] * 5
         lib.mcce_pipeline_submit_host.argtypes = [vp] * 5
+        lib.mcce_pipeline_submit.argtypes = [vp] * 6
         lib.mcce_pipeline_wait.argtypes = [vp]
         lib.mcce_cache_stats.argtypes = [vp, C.POINTER(Stats), C.POINTER(Stats)]
+        lib.mcce_calibrate_delta.argtypes = [vp, vp]
         lib.mcce_get_cache_state.argtypes = [vp, vp, vp, vp, C.POINTER(C.c_int64)]
         lib.mcce_get_grouping.argtypes = [vp, vp, vp]
         lib.mcce_lifetime_stats.argtypes = [vp, vp, vp]
@@ -129,12 +132,13 @@ class Engine:
 
     def __init__(self, *, L, E, K, J, n_shared, d, I, C_cap, S, lam, delta_mode=DELTA_RUNNING, renorm=1, dtype=BF16,
                  ffn_impl=FFN_AUTO, device=0, rerank_mode=RERANK_CACHE_PRIOR, max_rank=0, cum_threshold=0.0,
-                 track_lifetime=False, route_impl=ROUTE_AUTO):
+                 track_lifetime=False, route_impl=ROUTE_AUTO, deterministic=False, checked=False):
         if not torch.cuda.is_available():
             raise McceError("no CUDA device: this library has no CPU path")
         self.lib = load()
         self.cfg = Config(L, E, K, J, n_shared, d, I, C_cap, S, lam, delta_mode, renorm, dtype, dtype, ffn_impl,
-                          device, rerank_mode, max_rank, cum_threshold, int(track_lifetime), route_impl)
+                          device, rerank_mode, max_rank, cum_threshold, int(track_lifetime), route_impl,
+                          int(deterministic), int(checked))
         self.device = torch.device("cuda", device)
         nbytes = self.lib.mcce_workspace_bytes(C.byref(self.cfg))
         if nbytes == 0:
@@ -230,6 +234,14 @@ class Engine:
         _check(self.lib.mcce_pipeline_submit_host(self.ctx, _ptr(hidden_host), _ptr(y_host), _ptr(sel_host),
                                                   _stream()), self.ctx)
 
+    def pipeline_submit(self, hidden, y, sel=None, hidden_ready=None):
+        """The same with device tensors: hidden [L,S,d] must be complete (or `hidden_ready`, a torch.cuda.Event,
+        marks it); y [L,S,d] fp32 and sel [L,S,K] int32 are complete in the current stream's order.  Alternate
+        between two y tensors from call to call."""
+        assert hidden.is_cuda and y.is_cuda and y.dtype == torch.float32 and hidden.dtype == _tdtype(self.dtype)
+        ev = C.c_void_p(hidden_ready.cuda_event) if hidden_ready is not None else None
+        _check(self.lib.mcce_pipeline_submit(self.ctx, _ptr(hidden), _ptr(y), _ptr(sel), ev, _stream()), self.ctx)
+
     def pipeline_wait(self):
         _check(self.lib.mcce_pipeline_wait(self.ctx), self.ctx)
 
@@ -288,13 +300,12 @@ class Engine:
         return (n, mean, sd), per
 
     def calibrated_delta(self) -> np.ndarray:
-        """Per-layer logit range from the running statistics gathered so far (mean over streams of the
-        cumulative mean of max(z) - min(z)): the constants for a context in DELTA_FIXED mode, i.e. the
-        "estimate over a calibration set" variant of the paper's appendix on logit-range estimation."""
-        _, _, dsum, cnt = self.cache_state()
-        if cnt == 0:
-            raise McceError("no tokens routed yet: nothing to calibrate from")
-        return (dsum.astype(np.float64).mean(axis=1) / cnt).astype(np.float32)
+        """Per-layer logit range from the running statistics gathered so far (mcce_calibrate_delta): the
+        constants for a context in DELTA_FIXED mode, i.e. the "estimate over a calibration set" variant of
+        the paper's appendix on logit-range estimation."""
+        delta = np.empty(self.L, np.float32)
+        _check(self.lib.mcce_calibrate_delta(self.ctx, _ptr(delta)), self.ctx)
+        return delta
 
     def grouping(self):
         offsets = np.empty((self.L, self.E + 1), np.int32)

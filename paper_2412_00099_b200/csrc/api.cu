@@ -27,8 +27,15 @@ struct mcce_ctx {
   unsigned long long* life;
   float* sum_range;
   unsigned long long* stats_dev;
-  int32_t *offsets, *perm, *inv;
-  void *Xg, *H;
+  // grouping of a step: bucket offsets, permutation and its inverse, activations in expert order.  Two sets, so
+  // that the pipelined entry points can prepare one step while the experts of the previous one still read theirs
+  struct GroupBufs {
+    int32_t *offsets, *perm, *inv;
+    void* Xg;
+  } gb[2];
+  int last_slot;   // the set the latest forward used (mcce_get_grouping reads it)
+  int* group_counts;
+  void* H;
   float* O;
   void* stage_hidden;
   int32_t* stage_sel;
@@ -37,9 +44,9 @@ struct mcce_ctx {
   void* stage_hidden2;
   int32_t* stage_sel2;
   float *stage_w2, *stage_y2;
-  cudaStream_t pipe_in, pipe_out;   // copy streams, created on first use
-  cudaEvent_t pipe_h2d[2], pipe_done[2], pipe_compute[2];
-  int pipe_ready, pipe_slot, pipe_busy[2];
+  cudaStream_t pipe_in, pipe_out, pipe_prep;   // copy streams and the stream of routing + grouping, created on first use
+  cudaEvent_t pipe_h2d[2], pipe_done[2], pipe_compute[2], pipe_prep_done[2], pipe_sync;
+  int pipe_ready, pipe_slot, pipe_busy[2], pipe_used[2];
   // borrowed weights
   const float *Wr, *fixed_delta;
   const void *Wg, *Wu, *Wd, *shWg, *shWu, *shWd;
@@ -90,11 +97,12 @@ bool valid(const mcce_config* c) {
   if (c->rerank_mode == MCCE_RERANK_CUMSUM && !(c->cum_threshold >= 0.f)) return false;
   if (c->track_lifetime != 0 && c->track_lifetime != 1) return false;
   if (c->route_impl < MCCE_ROUTE_AUTO || c->route_impl > MCCE_ROUTE_FUSED) return false;
+  if ((c->deterministic != 0 && c->deterministic != 1) || (c->checked != 0 && c->checked != 1)) return false;
   return true;
 }
 
 struct Layout {
-  size_t stamp, ever, sum_range, miss, cold, err, stats, offsets, perm, inv, Xg, H, O, st_hidden, st_sel, st_w, st_y, st_hidden2, st_sel2, st_w2, st_y2,
+  size_t stamp, ever, sum_range, miss, cold, err, stats, offsets, perm, inv, offsets2, perm2, inv2, group_counts, Xg, Xg2, H, O, st_hidden, st_sel, st_w, st_y, st_hidden2, st_sel2, st_w2, st_y2,
       wr_terms, z_buf, z_ready, load_tok, life, total;
 };
 
@@ -119,11 +127,17 @@ Layout layout_of(const mcce_config& c) {
   o.offsets = take(L * (E + 1) * 4);
   o.perm = take(L * S * K * 4);
   o.inv = take(L * S * K * 4);
+  o.offsets2 = take(L * (E + 1) * 4);
+  o.perm2 = take(L * S * K * 4);
+  o.inv2 = take(L * S * K * 4);
+  o.group_counts = take((L * (size_t)group_chunks((int)S, (int)K) * E + L) * 4);   // histograms, then a ticket per layer
   o.Xg = take((L * S * K + 256) * d * esz);  // slack rows: tensor-core tiles read past a group's end
+  o.Xg2 = take((L * S * K + 256) * d * esz);
   o.H = take((rows + 256) * I * esz);
-  // per-pair expert outputs are only needed by the fp32-pipe path (the tensor path combines in its epilogue)
+  // per-pair expert outputs are needed by the fp32-pipe path and by the deterministic mode (otherwise the
+  // tensor path combines in its epilogue)
   const bool tensor_ffn = c.ffn_impl != MCCE_FFN_SIMT && tc_applicable(c);
-  o.O = take(tensor_ffn ? 0 : rows * d * 4);
+  o.O = take(tensor_ffn && !c.deterministic ? 0 : rows * d * 4);
   o.st_hidden = take(L * S * d * esz);
   o.st_sel = take(L * S * K * 4);
   o.st_w = take(L * S * K * 4);
@@ -134,10 +148,11 @@ Layout layout_of(const mcce_config& c) {
   o.st_y2 = take(L * S * d * 4);
   const bool rg = router_gemm_applicable(c);
   o.wr_terms = take(rg ? 3 * L * E * d * 2 : 0);
-  // logits of up to router_gemm_steps_max() tokens; the router-resident kernel writes one array per K part
-  const size_t z_slots = (size_t)router_gemm_steps_max() * (router_gemm_res_applicable(c) ? router_gemm_res_parts_max() : 1);
+  // logits of up to router_gemm_steps_max() tokens; the router-resident kernels write one array per K part, the
+  // fused one a further array with their sum
+  const size_t z_slots = (size_t)router_gemm_steps_max() * (router_gemm_res_applicable(c) ? router_gemm_res_parts_max() + 1 : 1);
   o.z_buf = take(rg ? z_slots * L * S * E * 4 : 0);
-  o.z_ready = take(rg ? (size_t)router_gemm_steps_max() * L * ((S + 127) / 128) * 4 : 0);   // counters of the fused kernel
+  o.z_ready = take(rg ? route_fused_counter_words((int)L, router_gemm_steps_max(), (int)S) * 4 : 0);   // counters of the fused kernel
   o.load_tok = take(c.track_lifetime ? L * S * E * 4 : 0);
   o.life = take(c.track_lifetime ? L * S * 3 * 8 : 0);
   o.total = p;
@@ -198,16 +213,26 @@ int timed(mcce_ctx* ctx, int kind, cudaStream_t st, F launch) {
     if (rc_ != MCCE_OK) return rc_;                             \
   } while (0)
 
-FfnParams ffn_params(const mcce_ctx* ctx, const void* hidden, const float* sel_w, float* y) {
+FfnParams ffn_params(const mcce_ctx* ctx, int slot, const void* hidden, const float* sel_w, float* y) {
   const mcce_config& c = ctx->cfg;
   FfnParams f;
   f.L = c.n_layers, f.S = c.n_streams, f.E = c.n_experts, f.K = c.top_k, f.n_sh = c.n_shared, f.l0 = 0;
   f.d = c.d_model, f.I = c.d_ff, f.bf16 = c.hidden_dtype == MCCE_BF16;
   f.hidden = hidden;
   f.Wg = ctx->Wg, f.Wu = ctx->Wu, f.Wd = ctx->Wd, f.shWg = ctx->shWg, f.shWu = ctx->shWu, f.shWd = ctx->shWd;
-  f.offsets = ctx->offsets, f.perm = ctx->perm, f.inv = ctx->inv, f.sel_w = sel_w;
-  f.Xg = ctx->Xg, f.H = ctx->H, f.O = ctx->O, f.y = y;
+  f.slot = slot;
+  f.offsets = ctx->gb[slot].offsets, f.perm = ctx->gb[slot].perm, f.inv = ctx->gb[slot].inv, f.sel_w = sel_w;
+  f.Xg = ctx->gb[slot].Xg, f.H = ctx->H, f.O = ctx->O, f.y = y;
   return f;
+}
+
+// Checked mode, after the routing launches of tokens whose logits lie in z (n floats; null when the route
+// kernel formed them itself and checked them on the way): logits finite, cache states consistent.
+int check_after_route(mcce_ctx* ctx, const float* z, size_t n, cudaStream_t st) {
+  const mcce_config& c = ctx->cfg;
+  if (z && n) CK(launch_check_finite(z, n, ctx->err + 2, st));
+  CK(launch_check_state(ctx->stamp, (size_t)c.n_layers * c.n_streams, c.n_experts, c.cache_capacity, ctx->err + 1, st));
+  return MCCE_OK;
 }
 
 }  // namespace
@@ -231,8 +256,12 @@ extern "C" int mcce_create(const mcce_config* cfg, void* workspace, size_t works
   ctx->sum_range = (float*)(w + lo.sum_range);
   ctx->miss = (uint32_t*)(w + lo.miss), ctx->cold = (uint32_t*)(w + lo.cold), ctx->err = (uint32_t*)(w + lo.err);
   ctx->stats_dev = (unsigned long long*)(w + lo.stats);
-  ctx->offsets = (int32_t*)(w + lo.offsets), ctx->perm = (int32_t*)(w + lo.perm), ctx->inv = (int32_t*)(w + lo.inv);
-  ctx->Xg = w + lo.Xg, ctx->H = w + lo.H, ctx->O = (float*)(w + lo.O);
+  ctx->gb[0].offsets = (int32_t*)(w + lo.offsets), ctx->gb[0].perm = (int32_t*)(w + lo.perm);
+  ctx->gb[0].inv = (int32_t*)(w + lo.inv), ctx->gb[0].Xg = w + lo.Xg;
+  ctx->gb[1].offsets = (int32_t*)(w + lo.offsets2), ctx->gb[1].perm = (int32_t*)(w + lo.perm2);
+  ctx->gb[1].inv = (int32_t*)(w + lo.inv2), ctx->gb[1].Xg = w + lo.Xg2;
+  ctx->group_counts = (int*)(w + lo.group_counts);
+  ctx->H = w + lo.H, ctx->O = (float*)(w + lo.O);
   ctx->stage_hidden = w + lo.st_hidden, ctx->stage_sel = (int32_t*)(w + lo.st_sel);
   ctx->stage_w = (float*)(w + lo.st_w), ctx->stage_y = (float*)(w + lo.st_y);
   ctx->stage_hidden2 = w + lo.st_hidden2, ctx->stage_sel2 = (int32_t*)(w + lo.st_sel2);
@@ -259,13 +288,17 @@ extern "C" int mcce_destroy(mcce_ctx* ctx) {
   if (!ctx) return MCCE_EINVAL;
   if (ctx->pipe_ready) {
     mcce_pipeline_wait(ctx);
+    cudaStreamSynchronize(ctx->pipe_prep);
     cudaStreamDestroy(ctx->pipe_in);
     cudaStreamDestroy(ctx->pipe_out);
+    cudaStreamDestroy(ctx->pipe_prep);
     for (int i = 0; i < 2; ++i) {
       cudaEventDestroy(ctx->pipe_h2d[i]);
       cudaEventDestroy(ctx->pipe_done[i]);
       cudaEventDestroy(ctx->pipe_compute[i]);
+      cudaEventDestroy(ctx->pipe_prep_done[i]);
     }
+    cudaEventDestroy(ctx->pipe_sync);
   }
   if (ctx->profiling)
     for (int i = 0; i < kMaxPairs; ++i) {
@@ -306,7 +339,7 @@ extern "C" int mcce_set_experts(mcce_ctx* ctx, const void* Wg, const void* Wu, c
     if ((uintptr_t)q % 16) return MCCE_EINVAL;
   ctx->Wg = Wg, ctx->Wu = Wu, ctx->Wd = Wd, ctx->shWg = shWg, ctx->shWu = shWu, ctx->shWd = shWd;
   if (ctx->use_tc) {
-    const int rc = tc_plan(ctx->cfg, Wg, Wu, Wd, shWg, shWu, shWd, ctx->Xg, ctx->H, &ctx->tc);
+    const int rc = tc_plan(ctx->cfg, Wg, Wu, Wd, shWg, shWu, shWd, ctx->gb[0].Xg, ctx->gb[1].Xg, ctx->H, &ctx->tc);
     if (rc != MCCE_OK) return rc;
   }
   return MCCE_OK;
@@ -362,6 +395,10 @@ extern "C" int mcce_route_step(mcce_ctx* ctx, int32_t n_steps, const void* hidde
   const mcce_config& c = ctx->cfg;
   if (hidden && !ctx->Wr) return MCCE_ESTATE;
   if (c.delta_mode == MCCE_DELTA_FIXED && !ctx->fixed_delta) return MCCE_ESTATE;
+  // rows of logits are read and written four floats at a time when E is a multiple of 4
+  const uintptr_t z_align = (c.n_experts & 3) ? 4 : 16;
+  if (((uintptr_t)logits_in % z_align) || ((uintptr_t)logits_out % z_align)) return MCCE_EINVAL;
+  if (hidden && ((uintptr_t)hidden % 16)) return MCCE_EINVAL;
   if (n_steps == 0) return MCCE_OK;
   // recency keys and the Delta count are 32-bit on the device
   const uint64_t last_key = (uint64_t)c.n_experts + (ctx->tok + n_steps) * (uint64_t)c.top_k + c.top_k + 1;
@@ -374,6 +411,7 @@ extern "C" int mcce_route_step(mcce_ctx* ctx, int32_t n_steps, const void* hidde
   p.Wr = ctx->Wr, p.fixed_delta = ctx->fixed_delta;
   p.stamp = ctx->stamp, p.ever = ctx->ever, p.sum_range = ctx->sum_range, p.miss = ctx->miss, p.cold = ctx->cold;
   p.load_tok = ctx->load_tok, p.life = ctx->life;
+  p.err_nonfinite = c.checked ? ctx->err + 2 : nullptr;
   const size_t LS_trace = (size_t)c.n_layers * c.n_streams;
   auto trace_at = [&](int t0, int nt) {   // where tokens [t0, t0+nt) of this call go in the trace buffer
     const int64_t pos = ctx->trace_pos + t0;
@@ -401,14 +439,19 @@ extern "C" int mcce_route_step(mcce_ctx* ctx, int32_t n_steps, const void* hidde
           return fe == cudaErrorCooperativeLaunchTooLarge ? cudaSuccess : fe;
         });
         if (rc_f != MCCE_OK) return rc_f;
-        if (fe == cudaSuccess) continue;
+        if (fe == cudaSuccess) {
+          if (c.checked) {
+            const int rc_c = check_after_route(ctx, ctx->z_buf, (size_t)ctx->rg.fused_parts * nt * LS * c.n_experts, st);
+            if (rc_c != MCCE_OK) return rc_c;
+          }
+          continue;
+        }
         // the device cannot hold the whole grid at once (it is shared with other work): two kernels from now on
         cudaGetLastError();
         ctx->rg.fused_ready = 0;
       }
       if (ctx->rg.res_ready) {
-        ks = ctx->rg.res_parts;
-        TIMED(MCCE_K_ROUTE_GEMM, st, router_gemm_res_launch(ctx->rg, c, h, nt, ctx->z_buf, ctx->err, st));
+        TIMED(MCCE_K_ROUTE_GEMM, st, router_gemm_res_launch(ctx->rg, c, h, nt, ctx->z_buf, &ks, ctx->err, st));
       } else {
         TIMED(MCCE_K_ROUTE_GEMM, st, router_gemm_launch(ctx->rg, c, h, nt, ctx->z_buf, &ks, ctx->err, st));
       }
@@ -419,6 +462,10 @@ extern "C" int mcce_route_step(mcce_ctx* ctx, int32_t n_steps, const void* hidde
       p.tok0 = (uint32_t)(ctx->tok + t0), p.cnt0 = (uint32_t)(ctx->delta_cnt + t0);
       trace_at(t0, nt);
       TIMED(MCCE_K_ROUTE, st, launch_route(p, st));
+      if (c.checked) {
+        const int rc_c = check_after_route(ctx, ctx->z_buf, (size_t)ks * nt * LS * c.n_experts, st);
+        if (rc_c != MCCE_OK) return rc_c;
+      }
     }
   } else {
     p.n_steps = n_steps, p.hidden = hidden, p.logits_in = logits_in, p.n_partials = 1, p.partial_stride = 0;
@@ -426,6 +473,10 @@ extern "C" int mcce_route_step(mcce_ctx* ctx, int32_t n_steps, const void* hidde
     p.tok0 = (uint32_t)ctx->tok, p.cnt0 = (uint32_t)ctx->delta_cnt;
     trace_at(0, n_steps);
     TIMED(MCCE_K_ROUTE, st, launch_route(p, st));
+    if (c.checked) {
+      const int rc_c = check_after_route(ctx, logits_in, logits_in ? (size_t)n_steps * c.n_layers * c.n_streams * c.n_experts : 0, st);
+      if (rc_c != MCCE_OK) return rc_c;
+    }
   }
   ctx->tok += n_steps;
   ctx->steps_since_reset += n_steps;
@@ -435,28 +486,51 @@ extern "C" int mcce_route_step(mcce_ctx* ctx, int32_t n_steps, const void* hidde
 }
 
 // Expert forward for model layers [l0, l0 + Ls): hidden, sel_idx, sel_w and y hold those layers only.  The
-// grouping, gathered rows and intermediates use the front of the context's buffers; only the expert weights
-// are addressed by model layer.
-static int forward_layers(mcce_ctx* ctx, int l0, int Ls, const void* hidden, const int32_t* sel_idx,
-                          const float* sel_w, float* y, cudaStream_t st) {
+// grouping, gathered rows and intermediates use the front of the context's buffers (set `slot` of the grouping
+// buffers); only the expert weights are addressed by model layer.  Two halves, which the pipelined entry points
+// put on different streams: the grouping pass with its row copy, and the expert kernels.
+static int group_layers(mcce_ctx* ctx, int slot, int Ls, const void* hidden, const int32_t* sel_idx, float* y,
+                        cudaStream_t st) {
   const mcce_config& c = ctx->cfg;
   GroupParams g;
   g.L = Ls, g.S = c.n_streams, g.E = c.n_experts, g.K = c.top_k;
-  g.sel_idx = sel_idx, g.offsets = ctx->offsets, g.perm = ctx->perm, g.inv = ctx->inv;
-  TIMED(MCCE_K_GROUP, st, launch_group(g, st));
-  FfnParams f = ffn_params(ctx, hidden, sel_w, y);
+  g.sel_idx = sel_idx, g.offsets = ctx->gb[slot].offsets, g.perm = ctx->gb[slot].perm, g.inv = ctx->gb[slot].inv;
+  g.err_index = ctx->err + 1;
+  int* tickets = ctx->group_counts + (size_t)c.n_layers * group_chunks(c.n_streams, c.top_k) * c.n_experts;
+  TIMED(MCCE_K_GROUP, st, launch_group(g, ctx->group_counts, tickets, st));
+  FfnParams f = ffn_params(ctx, slot, hidden, nullptr, y);
+  f.L = Ls;
+  // on the tensor path the down kernel adds w * E_i(x) into y itself: the grouping pass clears y on the way;
+  // in the deterministic mode it stores rows of O instead and the combine pass writes every element of y
+  const bool atomic_combine = ctx->use_tc && !c.deterministic;
+  TIMED(MCCE_K_GATHER, st, launch_place(g, f, ctx->group_counts, atomic_combine, st));
+  if (c.checked) CK(launch_check_group(g, st));
+  ctx->last_slot = slot;
+  return MCCE_OK;
+}
+
+static int expert_layers(mcce_ctx* ctx, int slot, int l0, int Ls, const void* hidden, const float* sel_w, float* y,
+                         cudaStream_t st) {
+  const mcce_config& c = ctx->cfg;
+  FfnParams f = ffn_params(ctx, slot, hidden, sel_w, y);
   f.L = Ls, f.l0 = l0;
-  // on the tensor path the down kernel adds w * E_i(x) into y itself: the gather pass clears y on the way
-  TIMED(MCCE_K_GATHER, st, launch_gather(f, ctx->use_tc != 0, st));
+  const bool atomic_combine = ctx->use_tc && !c.deterministic;
   if (ctx->use_tc) {
     TIMED(MCCE_K_FFN_UP, st, tc_launch_up(ctx->tc, f, ctx->err, st));
-    TIMED(MCCE_K_FFN_DOWN, st, tc_launch_down(ctx->tc, f, ctx->err, st));
+    TIMED(MCCE_K_FFN_DOWN, st, tc_launch_down(ctx->tc, f, !atomic_combine, ctx->err, st));
+    if (!atomic_combine) TIMED(MCCE_K_COMBINE, st, launch_combine(f, st));
   } else {
     TIMED(MCCE_K_FFN_UP, st, launch_ffn_simt_up(f, st));
     TIMED(MCCE_K_FFN_DOWN, st, launch_ffn_simt_down(f, st));
     TIMED(MCCE_K_COMBINE, st, launch_combine(f, st));
   }
   return MCCE_OK;
+}
+
+static int forward_layers(mcce_ctx* ctx, int l0, int Ls, const void* hidden, const int32_t* sel_idx,
+                          const float* sel_w, float* y, cudaStream_t st) {
+  const int rc = group_layers(ctx, 0, Ls, hidden, sel_idx, y, st);
+  return rc != MCCE_OK ? rc : expert_layers(ctx, 0, l0, Ls, hidden, sel_w, y, st);
 }
 
 extern "C" int mcce_moe_forward(mcce_ctx* ctx, const void* hidden, const int32_t* sel_idx, const float* sel_w,
@@ -490,14 +564,24 @@ static int route_one_layer(mcce_ctx* ctx, int l, const void* x, int32_t* sel, fl
   p.trace_avail = trace ? 1 : 0;
   p.sel_idx = sel, p.sel_w = w, p.logits_out = nullptr;
   p.tok0 = (uint32_t)ctx->tok, p.cnt0 = (uint32_t)ctx->delta_cnt;
+  p.err_nonfinite = c.checked ? ctx->err + 2 : nullptr;
+  int ks = 0;
   if (ctx->use_tc_router && ctx->rg.ready) {
-    int ks = 1;
-    TIMED(MCCE_K_ROUTE_GEMM, st, router_gemm_launch(ctx->rg, c, x, 1, ctx->z_buf, &ks, ctx->err, st, l, 1));
+    ks = 1;
+    // the kernel a one-layer context would launch for this layer
+    if (ctx->rg.res_ready)
+      TIMED(MCCE_K_ROUTE_GEMM, st, router_gemm_res_launch(ctx->rg, c, x, 1, ctx->z_buf, &ks, ctx->err, st, l, 1));
+    else
+      TIMED(MCCE_K_ROUTE_GEMM, st, router_gemm_launch(ctx->rg, c, x, 1, ctx->z_buf, &ks, ctx->err, st, l, 1));
     p.hidden = nullptr, p.logits_in = ctx->z_buf, p.n_partials = ks, p.partial_stride = S * E;
   } else {
     p.hidden = x, p.logits_in = nullptr, p.n_partials = 1, p.partial_stride = 0;
   }
   TIMED(MCCE_K_ROUTE, st, launch_route(p, st));
+  if (c.checked) {
+    if (ks) CK(launch_check_finite(ctx->z_buf, (size_t)ks * S * E, ctx->err + 2, st));
+    CK(launch_check_state(p.stamp, S, c.n_experts, c.cache_capacity, ctx->err + 1, st));
+  }
   return MCCE_OK;
 }
 
@@ -561,17 +645,24 @@ extern "C" int mcce_decode_step_host(mcce_ctx* ctx, const void* hidden_host, flo
   return MCCE_OK;
 }
 
-// ---- pipelined host entry point: two staging slots, a copy-in and a copy-out stream ---------------------
+// ---- pipelined entry points: two slots, routing + grouping of a step on a stream of their own -------------
+// Routing needs only the hidden states of its token and the cache state left by the previous token's routing,
+// not the previous token's experts.  So a step is split over streams: routing, grouping and the row copy of step
+// t + 1 run on the internal stream `pipe_prep` while the expert kernels of step t, which stream all the weights,
+// still run on the caller's stream; events order a step's two halves and guard the reuse of a slot's buffers.
 static int pipe_setup(mcce_ctx* ctx) {
   if (ctx->pipe_ready) return MCCE_OK;
   CK(cudaSetDevice(ctx->cfg.device));
   CK(cudaStreamCreateWithFlags(&ctx->pipe_in, cudaStreamNonBlocking));
   CK(cudaStreamCreateWithFlags(&ctx->pipe_out, cudaStreamNonBlocking));
+  CK(cudaStreamCreateWithFlags(&ctx->pipe_prep, cudaStreamNonBlocking));
   for (int i = 0; i < 2; ++i) {
     CK(cudaEventCreateWithFlags(&ctx->pipe_h2d[i], cudaEventDisableTiming));
     CK(cudaEventCreateWithFlags(&ctx->pipe_done[i], cudaEventDisableTiming));
     CK(cudaEventCreateWithFlags(&ctx->pipe_compute[i], cudaEventDisableTiming));
+    CK(cudaEventCreateWithFlags(&ctx->pipe_prep_done[i], cudaEventDisableTiming));
   }
+  CK(cudaEventCreateWithFlags(&ctx->pipe_sync, cudaEventDisableTiming));
   ctx->pipe_ready = 1;
   return MCCE_OK;
 }
@@ -587,9 +678,35 @@ extern "C" int mcce_pipeline_wait(mcce_ctx* ctx) {
   return MCCE_OK;
 }
 
+// One step in slot i: routing + grouping of `hidden` on pipe_prep (after `after_event`, if any, and after the
+// experts of the step that used the slot before), then the experts on st.  Records pipe_compute[i] on st.
+static int pipe_step(mcce_ctx* ctx, int i, const void* hidden, int32_t* sel, float* w, float* y, cudaEvent_t after_event,
+                     cudaStream_t st) {
+  const mcce_config& c = ctx->cfg;
+  if (!ctx->pipe_busy[0] && !ctx->pipe_busy[1]) {
+    // the pipeline is empty: whatever the caller's stream did to this context so far comes first
+    CK(cudaEventRecord(ctx->pipe_sync, st));
+    CK(cudaStreamWaitEvent(ctx->pipe_prep, ctx->pipe_sync, 0));
+  }
+  if (after_event) CK(cudaStreamWaitEvent(ctx->pipe_prep, after_event, 0));
+  if (ctx->pipe_used[i]) CK(cudaStreamWaitEvent(ctx->pipe_prep, ctx->pipe_compute[i], 0));
+  int rc = mcce_route_step(ctx, 1, hidden, nullptr, sel, w, nullptr, (void*)ctx->pipe_prep);
+  if (rc != MCCE_OK) return rc;
+  rc = group_layers(ctx, i, c.n_layers, hidden, sel, y, ctx->pipe_prep);
+  if (rc != MCCE_OK) return rc;
+  CK(cudaEventRecord(ctx->pipe_prep_done[i], ctx->pipe_prep));
+  CK(cudaStreamWaitEvent(st, ctx->pipe_prep_done[i], 0));
+  rc = expert_layers(ctx, i, 0, c.n_layers, hidden, w, y, st);
+  if (rc != MCCE_OK) return rc;
+  CK(cudaEventRecord(ctx->pipe_compute[i], st));
+  ctx->pipe_used[i] = 1;
+  return MCCE_OK;
+}
+
 extern "C" int mcce_pipeline_submit_host(mcce_ctx* ctx, const void* hidden_host, float* y_host, int32_t* sel_idx_host,
                                          void* cuda_stream) {
   if (!ctx || !hidden_host || !y_host) return MCCE_EINVAL;
+  if (!ctx->Wr || !ctx->Wg) return MCCE_ESTATE;
   int rc = pipe_setup(ctx);
   if (rc != MCCE_OK) return rc;
   const mcce_config& c = ctx->cfg;
@@ -607,16 +724,40 @@ extern "C" int mcce_pipeline_submit_host(mcce_ctx* ctx, const void* hidden_host,
   }
   CK(cudaMemcpyAsync(sh, hidden_host, LS * c.d_model * esz, cudaMemcpyHostToDevice, ctx->pipe_in));
   CK(cudaEventRecord(ctx->pipe_h2d[i], ctx->pipe_in));
-  CK(cudaStreamWaitEvent(st, ctx->pipe_h2d[i], 0));
-  rc = mcce_route_step(ctx, 1, sh, nullptr, ss, sw, nullptr, cuda_stream);
+  rc = pipe_step(ctx, i, sh, ss, sw, sy, ctx->pipe_h2d[i], st);
   if (rc != MCCE_OK) return rc;
-  rc = mcce_moe_forward(ctx, sh, ss, sw, sy, cuda_stream);
-  if (rc != MCCE_OK) return rc;
-  CK(cudaEventRecord(ctx->pipe_compute[i], st));
   CK(cudaStreamWaitEvent(ctx->pipe_out, ctx->pipe_compute[i], 0));
   CK(cudaMemcpyAsync(y_host, sy, LS * c.d_model * 4, cudaMemcpyDeviceToHost, ctx->pipe_out));
   if (sel_idx_host) CK(cudaMemcpyAsync(sel_idx_host, ss, LS * c.top_k * 4, cudaMemcpyDeviceToHost, ctx->pipe_out));
   CK(cudaEventRecord(ctx->pipe_done[i], ctx->pipe_out));
+  ctx->pipe_busy[i] = 1;
+  ctx->pipe_slot = i ^ 1;
+  return MCCE_OK;
+}
+
+extern "C" int mcce_pipeline_submit(mcce_ctx* ctx, const void* hidden, float* y, int32_t* sel_idx, void* hidden_ready,
+                                    void* cuda_stream) {
+  if (!ctx || !hidden || !y) return MCCE_EINVAL;
+  if (!ctx->Wr || !ctx->Wg) return MCCE_ESTATE;
+  if (((uintptr_t)hidden % 16) || ((uintptr_t)y % 16)) return MCCE_EINVAL;
+  int rc = pipe_setup(ctx);
+  if (rc != MCCE_OK) return rc;
+  const mcce_config& c = ctx->cfg;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  const size_t LS = (size_t)c.n_layers * c.n_streams;
+  const int i = ctx->pipe_slot;
+  int32_t* ss = i ? ctx->stage_sel2 : ctx->stage_sel;
+  float* sw = i ? ctx->stage_w2 : ctx->stage_w;
+  // steps of the host-buffer entry point that still use the slot's staging buffers come first
+  if (ctx->pipe_busy[i]) {
+    CK(cudaEventSynchronize(ctx->pipe_done[i]));
+    ctx->pipe_busy[i] = 0;
+  }
+  rc = pipe_step(ctx, i, hidden, ss, sw, y, (cudaEvent_t)hidden_ready, st);
+  if (rc != MCCE_OK) return rc;
+  if (sel_idx) CK(cudaMemcpyAsync(sel_idx, ss, LS * c.top_k * 4, cudaMemcpyDeviceToDevice, st));
+  // "left the device" for this entry point: the step's last work on the caller's stream
+  CK(cudaEventRecord(ctx->pipe_done[i], st));
   ctx->pipe_busy[i] = 1;
   ctx->pipe_slot = i ^ 1;
   return MCCE_OK;
@@ -643,7 +784,19 @@ extern "C" int mcce_cache_stats(mcce_ctx* ctx, mcce_stats* total, mcce_stats* pe
     total->steps += s.steps, total->selections += s.selections;
     total->misses += s.misses, total->cold_misses += s.cold_misses;
   }
-  return err[0] != 0 ? MCCE_ETIMEOUT : MCCE_OK;
+  return err[0] != 0 ? MCCE_ETIMEOUT : err[1] != 0 ? MCCE_EINDEX : err[2] != 0 ? MCCE_ENONFINITE : MCCE_OK;
+}
+
+extern "C" int mcce_calibrate_delta(mcce_ctx* ctx, float* delta) {
+  if (!ctx || !delta) return MCCE_EINVAL;
+  const mcce_config& c = ctx->cfg;
+  if (c.delta_mode != MCCE_DELTA_RUNNING || ctx->delta_cnt == 0) return MCCE_ESTATE;
+  CK(cudaSetDevice(c.device));
+  CK(cudaDeviceSynchronize());
+  float* out = (float*)ctx->stats_dev;   // L floats of the per-layer counter scratch (16 bytes per layer)
+  CK(launch_calibrate(ctx->sum_range, c.n_layers, c.n_streams, (double)ctx->delta_cnt, out, 0));
+  CK(cudaMemcpy(delta, out, (size_t)c.n_layers * 4, cudaMemcpyDeviceToHost));
+  return MCCE_OK;
 }
 
 extern "C" int mcce_get_cache_state(mcce_ctx* ctx, int32_t* order, uint8_t* ever, float* delta_sum,
@@ -708,8 +861,9 @@ extern "C" int mcce_get_grouping(mcce_ctx* ctx, int32_t* offsets, int32_t* perm)
   const mcce_config& c = ctx->cfg;
   CK(cudaSetDevice(c.device));
   CK(cudaDeviceSynchronize());
-  CK(cudaMemcpy(offsets, ctx->offsets, (size_t)c.n_layers * (c.n_experts + 1) * 4, cudaMemcpyDeviceToHost));
-  CK(cudaMemcpy(perm, ctx->perm, (size_t)c.n_layers * c.n_streams * c.top_k * 4, cudaMemcpyDeviceToHost));
+  const mcce_ctx::GroupBufs& gb = ctx->gb[ctx->last_slot];
+  CK(cudaMemcpy(offsets, gb.offsets, (size_t)c.n_layers * (c.n_experts + 1) * 4, cudaMemcpyDeviceToHost));
+  CK(cudaMemcpy(perm, gb.perm, (size_t)c.n_layers * c.n_streams * c.top_k * 4, cudaMemcpyDeviceToHost));
   return MCCE_OK;
 }
 
@@ -779,6 +933,10 @@ extern "C" const char* mcce_strerror(int code) {
              "overflow (call mcce_reset)";
     case MCCE_ECUDA: return "CUDA call failed (see mcce_last_cuda_error)";
     case MCCE_ETIMEOUT: return "a bounded wait inside a kernel gave up";
+    case MCCE_EINDEX:
+      return "an expert id outside [0, E) was skipped by the grouping pass, or a consistency check of the checked "
+             "mode failed (grouping position, cache occupancy or recency keys)";
+    case MCCE_ENONFINITE: return "a router logit was NaN or infinite (checked mode)";
     case MCCE_ELIMIT:
       return "the cache state of this configuration exceeds the fixed 4 MiB array of mcce_route_trace_static "
              "(use mcce_create with a workspace instead)";

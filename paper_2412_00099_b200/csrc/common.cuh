@@ -42,14 +42,23 @@ struct RouteParams {
   float* logits_out;         // [n_steps,L,S,E] or null
   uint32_t tok0;             // tokens already processed since the last reset
   uint32_t cnt0;             // tokens already folded into the running Delta
+  uint32_t* err_nonfinite;   // checked mode: set by the kernel that forms its own logits when one is not finite; else null
 };
+
+// Bits of the context's index-error word (the second word of its error block; the first is the code of a
+// bounded wait that gave up, the third is set when the checked mode meets a non-finite logit).
+constexpr uint32_t kErrBadExpertId = 1u;   // sel_idx entry outside [0, E): the pair was skipped
+constexpr uint32_t kErrBadPosition = 2u;   // checked mode: offsets not monotone or a position outside [0, S*K)
+constexpr uint32_t kErrOverCapacity = 4u;  // checked mode: more than C resident experts in a (stream, layer)
+constexpr uint32_t kErrDuplicateKey = 8u;  // checked mode: two resident experts with the same recency key
 
 struct GroupParams {
   int L, S, E, K;
   const int32_t* sel_idx;  // [L,S,K]
   int32_t* offsets;        // [L,E+1]
   int32_t* perm;           // [L,S*K] position -> pair
-  int32_t* inv;            // [L,S*K] pair -> position
+  int32_t* inv;            // [L,S*K] pair -> position, -1 for a pair whose expert id is out of range
+  uint32_t* err_index;     // index-error word of the context
 };
 
 // Rows of the activation / intermediate / output buffers: routed pairs first, [l][pos], then the
@@ -57,6 +66,7 @@ struct GroupParams {
 struct FfnParams {
   int L, S, E, K, n_sh, d, I;
   int l0;  // model layer of local layer 0: only the weights are indexed by model layer, everything else is local
+  int slot;  // which of the two sets of grouping buffers (and of their tensor maps) this step uses
   int bf16;
   const void* hidden;  // [L,S,d]
   const void *Wg, *Wu, *Wd, *shWg, *shWu, *shWd;
@@ -80,6 +90,7 @@ struct RouterGemmPlan {
   uint64_t hidden_rows_res;
   int ready;
   int res_ready, res_parts;   // K parts (= partial logit arrays) of the router-resident kernel
+  int res_parts_single;       // the same for a launch of one layer at a time
   int fused_ready, fused_parts;   // the same for the kernel that also runs the routing tail (route_fused.cu)
 };
 bool router_gemm_applicable(const mcce_config& c);
@@ -92,9 +103,10 @@ bool router_gemm_res_applicable(const mcce_config& c);
 int router_gemm_res_parts_max();
 int router_gemm_res_plan(const mcce_config& c, void* terms, RouterGemmPlan* plan);
 cudaError_t router_gemm_res_launch(RouterGemmPlan& plan, const mcce_config& c, const void* hidden, int n_steps,
-                                   float* Z, uint32_t* err, cudaStream_t st);
+                                   float* Z, int* k_parts, uint32_t* err, cudaStream_t st, int l0 = 0, int n_layers = 0);
 
 int route_fused_plan(const mcce_config& c, RouterGemmPlan* plan);
+size_t route_fused_counter_words(int n_layers, int n_steps, int n_streams);
 cudaError_t route_fused_launch(RouterGemmPlan& plan, const mcce_config& c, const void* hidden, int n_steps, float* Z,
                                uint32_t* ready, RouteParams p, uint32_t* err, cudaStream_t st);
 
@@ -103,14 +115,21 @@ cudaError_t launch_wait_timeout_selftest(uint32_t* err, unsigned long long limit
 cudaError_t launch_route(const RouteParams& p, cudaStream_t st);   // picks the thread-per-stream kernel where it applies
 bool route_thread_applicable(const RouteParams& p);
 cudaError_t launch_route_thread(const RouteParams& p, cudaStream_t st);
-cudaError_t launch_group(const GroupParams& p, cudaStream_t st);
-cudaError_t launch_gather(const FfnParams& p, bool zero_y, cudaStream_t st);
+int group_chunks(int S, int K);   // CTAs per layer of the grouping kernels (= histograms per layer)
+cudaError_t launch_group(const GroupParams& p, int* counts /*[L][group_chunks][E]*/, int* tickets /*[L], zero*/,
+                         cudaStream_t st);
+cudaError_t launch_place(const GroupParams& p, const FfnParams& f, const int* counts, bool zero_y, cudaStream_t st);
 cudaError_t launch_ffn_simt_up(const FfnParams& p, cudaStream_t st);
 cudaError_t launch_ffn_simt_down(const FfnParams& p, cudaStream_t st);
 cudaError_t launch_combine(const FfnParams& p, cudaStream_t st);
 cudaError_t launch_residual(const void* x_in, const float* y, void* x_out, size_t n, bool bf16, cudaStream_t st);
 cudaError_t launch_stats(const uint32_t* miss, const uint32_t* cold, unsigned long long* out, int L, int S,
                          cudaStream_t st);
+cudaError_t launch_check_group(const GroupParams& p, cudaStream_t st);
+cudaError_t launch_check_state(const uint32_t* stamp, size_t n_pairs, int E, int C, uint32_t* err_index,
+                               cudaStream_t st);
+cudaError_t launch_check_finite(const float* z, size_t n, uint32_t* err_nonfinite, cudaStream_t st);
+cudaError_t launch_calibrate(const float* sum_range, int L, int S, double count, float* out, cudaStream_t st);
 
 __device__ __forceinline__ float bf16_to_f32(__nv_bfloat16 v) { return __bfloat162float(v); }
 

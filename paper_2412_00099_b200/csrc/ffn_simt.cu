@@ -167,6 +167,7 @@ __global__ void combine_kernel(const FfnParams p) {
   for (int j = 4 * threadIdx.x; j < p.d; j += 4 * blockDim.x) {
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int k = 0; k < p.K; ++k) {
+      if (pos[k] < 0) continue;   // pair skipped by the grouping pass (expert id out of range)
       const float4 o = __ldg((const float4*)(p.O + ((size_t)l * P + pos[k]) * p.d + j));
       acc.x = fmaf(w[k], o.x, acc.x);
       acc.y = fmaf(w[k], o.y, acc.y);

@@ -14,8 +14,10 @@
 // stages, warp 1 issues tcgen05.mma into one of two TMEM accumulator buffers, warps 2-5 drain the other
 // buffer with tcgen05.ld and apply the epilogue: SwiGLU and a bf16 store of H (up), or the weighted
 // combine of Eq. 1 straight into y with fp32 atomic adds (down; y is zeroed first, and since the order
-// of a stream's K + shared addends is not fixed, the last bits of y may differ from run to run).  Every wait on an mbarrier is bounded:
-// on a timeout the CTA records an error word, stops, releases its TMEM and returns.
+// of a stream's K + shared addends is not fixed, the last bits of y may differ from run to run).  In the
+// deterministic mode the down kernel instead stores one fp32 row per (stream, slot) and a second pass adds
+// them in slot order.  Every wait on an mbarrier is bounded: on a timeout the CTA records an error word,
+// stops, releases its TMEM and returns.
 #include <cuda.h>
 
 #include "ffn_tc.cuh"
@@ -48,6 +50,16 @@ struct Cfg {
   static constexpr size_t kSmemBytes = (size_t)kStages * kStageBytes + 1024 /*align*/ + 256 /*barriers*/;
 };
 
+// The tensor core's fp32 accumulate truncates, which over the hundreds of accumulation steps of a long reduction
+// adds up to a relative bias of about 1e-5 -- enough to flip the bf16 rounding of H in a few dozen places per
+// token and expert.  A pass over few tokens therefore spreads its K-slabs round-robin over up to four accumulator
+// sets (each in its own TMEM columns, as many as fit beside each other), and the epilogue adds the sets in
+// round-to-nearest fp32: each accumulator then sees a quarter of the steps.
+__host__ __device__ __forceinline__ int acc_sets(int n_pad, int KT) {
+  const int s = n_pad <= 32 ? 4 : n_pad <= 64 ? 2 : 1;
+  return s < KT ? s : (KT >= 2 ? 2 : 1);
+}
+
 struct TcArgs {
   int L, S, E, K, n_sh, d, I;
   int l0;                // model layer of local layer 0 (weights are indexed by model layer)
@@ -57,6 +69,7 @@ struct TcArgs {
   const float* sel_w;    // [L, S, K]
   __nv_bfloat16* H;
   float* y;              // [L, S, d], zeroed before the down kernel; receives w * E_i(x) by fp32 atomic adds
+  float* O;              // [rows, d] expert outputs per (stream, slot), deterministic mode only
   uint32_t* err;
 };
 
@@ -98,7 +111,7 @@ __device__ __forceinline__ Item decode(const TcArgs& a, int w) {
     const int g = wl / RT;
     it.col0 = (wl % RT) * span;
     const int o0 = __ldg(a.offsets + (size_t)l * (a.E + 1) + g);
-    it.m = __ldg(a.offsets + (size_t)l * (a.E + 1) + g + 1) - o0;
+    it.m = min(max(__ldg(a.offsets + (size_t)l * (a.E + 1) + g + 1) - o0, 0), P);   // never beyond a layer's pairs
     it.shared = false;
     it.wrow = ((a.l0 + l) * a.E + g) * rows + it.col0;
     it.xrow = l * P + o0;
@@ -117,7 +130,9 @@ __device__ __forceinline__ Item decode(const TcArgs& a, int w) {
   return it;
 }
 
-template <bool UP>
+// UP: gate/up projection.  Otherwise the down projection, which either adds w * E_i(x) into y (ROWS_OUT
+// false) or stores the unweighted expert outputs row by row into O (ROWS_OUT true, deterministic mode).
+template <bool UP, bool ROWS_OUT>
 __global__ void __launch_bounds__(kThreads, 1)
 ffn_tc_kernel(const __grid_constant__ TcMaps maps, const TcArgs a) {
   using C = Cfg<UP>;
@@ -199,6 +214,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, const TcArgs a) {
         for (int c0 = 0; c0 < it.m && alive; c0 += kNMax, ++acc_iter) {
           const uint32_t n = (uint32_t)(min(kNMax, it.m - c0) + 15) & ~15u;
           const uint32_t idesc = instr_desc(n);
+          const int sets = acc_sets((int)n, KT);
           const uint32_t buf = acc_iter & 1u, acc_phase = (acc_iter >> 1) & 1u;
           if (!mbar_wait(bar_tempty + 8 * buf, acc_phase ^ 1u, abort_flag, a.err, 2u)) {
             alive = false;
@@ -215,11 +231,12 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, const TcArgs a) {
             const uint32_t sa = smem_base + stage * C::kStageBytes;
             const uint32_t sb = sa + 2 * kABytes;
 #pragma unroll
+            const uint32_t ds = d0 + (uint32_t)(kt % sets) * n;   // this slab's accumulator set
             for (int k = 0; k < kTileK / 16; ++k) {
-              const uint32_t acc = (kt > 0 || k > 0) ? 1u : 0u;
+              const uint32_t acc = (kt >= sets || k > 0) ? 1u : 0u;
               const uint64_t bd = smem_desc(sb + k * 32);
-              umma_bf16(d0, smem_desc(sa + k * 32), bd, idesc, acc);
-              if (it.ntile == 2) umma_bf16(d0 + kNMax, smem_desc(sa + kABytes + k * 32), bd, idesc, acc);
+              umma_bf16(ds, smem_desc(sa + k * 32), bd, idesc, acc);
+              if (it.ntile == 2) umma_bf16(ds + kNMax, smem_desc(sa + kABytes + k * 32), bd, idesc, acc);
             }
             umma_commit(bar_empty + 8 * stage);   // frees the stage once these MMAs have read it
             if (++stage == C::kStages) stage = 0, phase ^= 1u;
@@ -249,18 +266,42 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, const TcArgs a) {
         }
         tc_fence_after();
         const uint32_t t0 = tmem_base + lane_addr + buf * C::kAccCols;
+        const int sets = acc_sets(n, KT);
+        // sum of the accumulator sets of 16 columns starting at column `col0` of the buffer
+        auto ld_sets = [&](uint32_t col0, float (&v)[16]) {
+          tmem_ld16(t0 + col0, v);
+          for (int sidx = 1; sidx < sets; ++sidx) {
+            float w[16];
+            tmem_ld16(t0 + col0 + (uint32_t)(sidx * n), w);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 16; ++j) v[j] = __fadd_rn(v[j], w[j]);
+          }
+        };
         for (int n0 = 0; n0 < n; n0 += 16) {
           float g[16];
-          tmem_ld16(t0 + n0, g);
+          ld_sets((uint32_t)n0, g);
           if (UP) {
             float u[16];
-            tmem_ld16(t0 + kNMax + n0, u);
+            ld_sets((uint32_t)(kNMax + n0), u);
             tmem_ld_wait();
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
               if (n0 + j < ntok) {
                 const float h = __fdividef(g[j], 1.f + __expf(-g[j])) * u[j];
                 a.H[(it.orow + c0 + n0 + j) * a.I + col] = __float2bfloat16_rn(h);
+              }
+            }
+          } else if (ROWS_OUT) {
+            float g2[16];
+            if (it.ntile == 2) ld_sets((uint32_t)(kNMax + n0), g2);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              if (n0 + j < ntok) {
+                float* o = a.O + (it.orow + c0 + n0 + j) * a.d + col;
+                o[0] = g[j];
+                if (it.ntile == 2) o[kTileM] = g2[j];
               }
             }
           } else {
@@ -280,7 +321,7 @@ ffn_tc_kernel(const __grid_constant__ TcMaps maps, const TcArgs a) {
               }
             }
             float g2[16];
-            if (it.ntile == 2) tmem_ld16(t0 + kNMax + n0, g2);   // second row range: columns col + 128
+            if (it.ntile == 2) ld_sets((uint32_t)(kNMax + n0), g2);   // second row range: columns col + 128
             tmem_ld_wait();
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
@@ -327,18 +368,19 @@ bool make_map(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, ui
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <bool UP>
+template <bool UP, bool ROWS_OUT>
 cudaError_t launch(const TcMaps& maps, const FfnParams& p, uint32_t* err, cudaStream_t st) {
   static int cache[64] = {0};   // one per instantiation of this launcher, i.e. per kernel
   int sms = 0;
-  cudaError_t e0 = sm_count_and_smem_optin(ffn_tc_kernel<UP>, Cfg<UP>::kSmemBytes, cache, &sms);
+  cudaError_t e0 = sm_count_and_smem_optin(ffn_tc_kernel<UP, ROWS_OUT>, Cfg<UP>::kSmemBytes, cache, &sms);
   if (e0 != cudaSuccess) return e0;
   TcArgs a;
   a.L = p.L, a.S = p.S, a.E = p.E, a.K = p.K, a.n_sh = p.n_sh, a.d = p.d, a.I = p.I, a.l0 = p.l0;
   a.n_items = p.L * items_per_layer(p.E, p.n_sh, p.S, UP ? p.I / kTileM : (p.d / kTileM + 1) / 2);
-  a.offsets = p.offsets, a.perm = p.perm, a.sel_w = p.sel_w, a.H = (__nv_bfloat16*)p.H, a.y = p.y, a.err = err;
+  a.offsets = p.offsets, a.perm = p.perm, a.sel_w = p.sel_w, a.H = (__nv_bfloat16*)p.H, a.y = p.y, a.O = p.O;
+  a.err = err;
   const int grid = a.n_items < sms ? a.n_items : sms;
-  ffn_tc_kernel<UP><<<grid, kThreads, Cfg<UP>::kSmemBytes, st>>>(maps, a);
+  ffn_tc_kernel<UP, ROWS_OUT><<<grid, kThreads, Cfg<UP>::kSmemBytes, st>>>(maps, a);
   return cudaGetLastError();
 }
 
@@ -350,7 +392,7 @@ bool tc_applicable(const mcce_config& c) {
 }
 
 int tc_plan(const mcce_config& c, const void* Wg, const void* Wu, const void* Wd, const void* shWg, const void* shWu,
-            const void* shWd, void* Xg, void* H, TcPlan* plan) {
+            const void* shWd, void* Xg0, void* Xg1, void* H, TcPlan* plan) {
   const uint64_t L = c.n_layers, E = c.n_experts, S = c.n_streams, K = c.top_k, nsh = c.n_shared;
   const uint64_t d = c.d_model, I = c.d_ff;
   const uint64_t rows = L * S * K + L * nsh * S;
@@ -359,33 +401,35 @@ int tc_plan(const mcce_config& c, const void* Wg, const void* Wu, const void* Wd
   if (nsh)
     ok = ok && make_map(&plan->sh_gate, shWg, L * nsh * I, d, kTileM) &&
          make_map(&plan->sh_up, shWu, L * nsh * I, d, kTileM) && make_map(&plan->sh_down, shWd, L * nsh * d, I, kTileM);
-  ok = ok && make_map(&plan->x_routed, Xg, L * S * K + 256, d, kXBox) && make_map(&plan->h_all, H, rows + 256, I, kXBox);
-  plan->hidden_ptr = nullptr;
-  plan->hidden_rows = 0;
+  ok = ok && make_map(&plan->x_routed[0], Xg0, L * S * K + 256, d, kXBox) &&
+       make_map(&plan->x_routed[1], Xg1, L * S * K + 256, d, kXBox) && make_map(&plan->h_all, H, rows + 256, I, kXBox);
+  plan->hidden_ptr[0] = plan->hidden_ptr[1] = nullptr;
+  plan->hidden_rows[0] = plan->hidden_rows[1] = 0;
   plan->ready = ok;
   return ok ? MCCE_OK : MCCE_ECUDA;
 }
 
 cudaError_t tc_launch_up(TcPlan& plan, const FfnParams& p, uint32_t* err_flag, cudaStream_t st) {
   if (!plan.ready) return cudaErrorNotReady;
-  if (p.n_sh && (plan.hidden_ptr != p.hidden || plan.hidden_rows != (uint64_t)p.L * p.S)) {
-    if (!make_map(&plan.x_hidden, p.hidden, (uint64_t)p.L * p.S, p.d, kXBox)) return cudaErrorInvalidValue;
-    plan.hidden_ptr = p.hidden;
-    plan.hidden_rows = (uint64_t)p.L * p.S;
+  const int sl = p.slot & 1;
+  if (p.n_sh && (plan.hidden_ptr[sl] != p.hidden || plan.hidden_rows[sl] != (uint64_t)p.L * p.S)) {
+    if (!make_map(&plan.x_hidden[sl], p.hidden, (uint64_t)p.L * p.S, p.d, kXBox)) return cudaErrorInvalidValue;
+    plan.hidden_ptr[sl] = p.hidden;
+    plan.hidden_rows[sl] = (uint64_t)p.L * p.S;
   }
   TcMaps m;
-  m.w0 = plan.w_gate, m.w1 = plan.w_up, m.x = plan.x_routed;
+  m.w0 = plan.w_gate, m.w1 = plan.w_up, m.x = plan.x_routed[sl];
   m.sw0 = p.n_sh ? plan.sh_gate : plan.w_gate, m.sw1 = p.n_sh ? plan.sh_up : plan.w_up;
-  m.xs = p.n_sh ? plan.x_hidden : plan.x_routed;
-  return launch<true>(m, p, err_flag, st);
+  m.xs = p.n_sh ? plan.x_hidden[sl] : plan.x_routed[sl];
+  return launch<true, false>(m, p, err_flag, st);
 }
 
-cudaError_t tc_launch_down(TcPlan& plan, const FfnParams& p, uint32_t* err_flag, cudaStream_t st) {
+cudaError_t tc_launch_down(TcPlan& plan, const FfnParams& p, bool rows_out, uint32_t* err_flag, cudaStream_t st) {
   if (!plan.ready) return cudaErrorNotReady;
   TcMaps m;
   m.w0 = plan.w_down, m.w1 = plan.w_down, m.x = plan.h_all, m.xs = plan.h_all;
   m.sw0 = p.n_sh ? plan.sh_down : plan.w_down, m.sw1 = m.sw0;
-  return launch<false>(m, p, err_flag, st);
+  return rows_out ? launch<false, true>(m, p, err_flag, st) : launch<false, false>(m, p, err_flag, st);
 }
 
 }  // namespace mcce

@@ -129,6 +129,12 @@ __global__ void __launch_bounds__(kWarps * 32, HIDDEN ? 1 : 4) route_kernel(cons
     }
     if (!active) continue;
 
+    if (HIDDEN && p.err_nonfinite != nullptr) {   // checked mode: these logits exist nowhere else
+      bool bad = false;
+#pragma unroll
+      for (int i = 0; i < NE; ++i) bad |= lane + 32 * i < E && !isfinite(zr[i]);
+      if (bad) atomicOr(p.err_nonfinite, 1u);
+    }
     if (p.logits_out != nullptr) {
 #pragma unroll
       for (int i = 0; i < NE; ++i)
@@ -193,7 +199,8 @@ __global__ void __launch_bounds__(kWarps * 32, HIDDEN ? 1 : 4) route_kernel(cons
       }
       int M = p.max_rank;
       if (p.rerank_mode == MCCE_RERANK_CUMSUM) {
-        // Algorithm 2: walk down the ranking, summing router probabilities until they reach the threshold
+        // Sec. 3.2 / Algorithm 2: M is the first number of ranks whose router probabilities, added rank by rank
+        // in fp32, reach the threshold (all E if they never do)
         float pr[NE], loc = 0.f;
 #pragma unroll
         for (int i = 0; i < NE; ++i) {
@@ -201,17 +208,15 @@ __global__ void __launch_bounds__(kWarps * 32, HIDDEN ? 1 : 4) route_kernel(cons
           loc += pr[i];
         }
         const float inv_all = warp_sum(loc);
-        float p_cum = 0.f;
-        M = 0;
-        while (p_cum < p.cum_threshold && M < E) {
+        float mass = 0.f;
+        for (M = 0; M < E && !(mass >= p.cum_threshold); ++M) {
+          // the probability of the expert of rank M sits in exactly one lane
           float wv = 0.f;
-          bool own = false;   // exactly one lane holds the expert of rank M
+          bool own = false;
 #pragma unroll
           for (int i = 0; i < NE; ++i)
             if (lane + 32 * i < E && rk[i] == (uint32_t)M) wv = pr[i] / inv_all, own = true;
-          wv = __shfl_sync(kFull, wv, __ffs(__ballot_sync(kFull, own)) - 1);
-          p_cum = __fadd_rn(p_cum, wv);
-          ++M;
+          mass = __fadd_rn(mass, __shfl_sync(kFull, wv, __ffs(__ballot_sync(kFull, own)) - 1));
         }
       }
 #pragma unroll
@@ -402,6 +407,75 @@ __global__ void stats_kernel(const uint32_t* miss, const uint32_t* cold, unsigne
     out[2 * l] = tm;
     out[2 * l + 1] = tc;
   }
+}
+
+// Logit range from a calibration set (appendix "Logit Range Estimation"): per layer, the mean over the streams
+// of the running estimate of Eq. 8, out[l] = (sum_s sum_range[l][s] / S) / count, in double precision (the
+// sum of a few hundred fp32 values is exact there, so the order of the additions does not matter), rounded
+// once to fp32.  One CTA per layer.
+__global__ void calibrate_kernel(const float* sum_range, int S, double count, float* out) {
+  __shared__ double part[256];
+  const int l = blockIdx.x;
+  double acc = 0.0;
+  for (int s = threadIdx.x; s < S; s += blockDim.x) acc += (double)sum_range[(size_t)l * S + s];
+  part[threadIdx.x] = acc;
+  __syncthreads();
+  for (int w = blockDim.x / 2; w > 0; w >>= 1) {
+    if ((int)threadIdx.x < w) part[threadIdx.x] += part[threadIdx.x + w];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) out[l] = (float)(part[0] / (double)S / count);
+}
+
+cudaError_t launch_calibrate(const float* sum_range, int L, int S, double count, float* out, cudaStream_t st) {
+  calibrate_kernel<<<L, 256, 0, st>>>(sum_range, S, count, out);
+  return cudaGetLastError();
+}
+
+// Checked mode, after a routing launch: one warp per (layer, stream) verifies that at most C experts are
+// resident and that the recency keys of the resident experts are distinct (the LRU order is then total).
+__global__ void check_state_kernel(const uint32_t* stamp, size_t n_pairs, int E, int C, uint32_t* err_index) {
+  const size_t pair = (size_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (pair >= n_pairs) return;
+  const int lane = threadIdx.x & 31;
+  const uint32_t* st = stamp + pair * E;
+  int resident = 0;
+  bool dup = false;
+  for (int e0 = 0; e0 < E; e0 += 32) {
+    const uint32_t mine = e0 + lane < E ? st[e0 + lane] : 0u;
+    resident += __popc(__ballot_sync(kFull, mine != 0u));
+    // against every expert of this and the later blocks (each unordered pair is visited once)
+    for (int f0 = e0; f0 < E; f0 += 32) {
+      const uint32_t other = f0 + lane < E ? st[f0 + lane] : 0u;
+      for (int j = 0; j < 32; ++j) {
+        const uint32_t o = __shfl_sync(kFull, other, j);
+        dup |= mine != 0u && o == mine && f0 + j != e0 + lane;
+      }
+    }
+  }
+  if (__any_sync(kFull, dup) && lane == 0) atomicOr(err_index, kErrDuplicateKey);
+  if (resident > C && lane == 0) atomicOr(err_index, kErrOverCapacity);
+}
+
+cudaError_t launch_check_state(const uint32_t* stamp, size_t n_pairs, int E, int C, uint32_t* err_index,
+                               cudaStream_t st) {
+  const int wpb = 8;
+  check_state_kernel<<<(unsigned)((n_pairs + wpb - 1) / wpb), wpb * 32, 0, st>>>(stamp, n_pairs, E, C, err_index);
+  return cudaGetLastError();
+}
+
+// Checked mode: sets *err_nonfinite when any of the n logits is NaN or infinite.
+__global__ void check_finite_kernel(const float* z, size_t n, uint32_t* err_nonfinite) {
+  bool bad = false;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+    bad |= !isfinite(z[i]);
+  if (bad) atomicOr(err_nonfinite, 1u);
+}
+
+cudaError_t launch_check_finite(const float* z, size_t n, uint32_t* err_nonfinite, cudaStream_t st) {
+  const size_t blocks = (n + 255) / 256;
+  check_finite_kernel<<<(unsigned)(blocks > 1184 ? 1184 : blocks), 256, 0, st>>>(z, n, err_nonfinite);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_stats(const uint32_t* miss, const uint32_t* cold, unsigned long long* out, int L, int S,

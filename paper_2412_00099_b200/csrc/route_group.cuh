@@ -99,18 +99,31 @@ struct Pre {
   uint32_t topj;
 };
 
+// How the logits of a token reach the registers.
+constexpr int kLoadDirect = 0;     // loaded when the token's turn comes (after sync.wait(t))
+constexpr int kPrefetchAll = 1;    // every token is there already: the next token's logits are requested while
+                                   // the current one is routed
+constexpr int kPrefetchReady = 2;  // tokens appear while the kernel runs: the next token's logits are requested
+                                   // early if sync.ready(t + 1) says they are there, else after sync.wait(t + 1)
+
+// For callers whose logits are all there before the launch.
+struct AllPresent {
+  __device__ __forceinline__ bool wait(int) const { return true; }
+  __device__ __forceinline__ bool ready(int) const { return true; }
+};
+
 // Routes the p.n_steps tokens of stream s_raw of layer l.  All 32 lanes of a warp must call this together
 // (groups past the last stream run on stream 0's data and store nothing).  `sub` is the lane's index in its
-// group.  wait(t) is called by every lane before the logits of token t are read and returns false to give up
-// (the same answer in all lanes of a warp).
+// group.  sync.wait(t) is called by every lane before the logits of token t are read and returns false to give
+// up; sync.ready(t) asks without waiting whether they can be read (both: the same answer in all lanes of a warp).
 //
 // A token's work has a part that does not depend on the cache (logits, range statistic, bias, top-J: stage A)
 // and a part that does (promotion, top-K, misses, LRU: stage B); only B is a chain from token to token.
-// PF: the next token's partial logits are requested while the current token is routed; this assumes that all
-// tokens are there already (a wait() that is always true).
-template <int G, int KMAX, bool PF, bool COHERENT, typename Wait>
+// With a prefetching MODE up to NP partial logit arrays of the next token are held in registers.
+template <int G, int KMAX, int MODE, int NP, bool COHERENT, typename Sync>
 __device__ __forceinline__ void route_group_streams(const RouteParams& p, const int l, const int s_raw, const int sub,
-                                                    Wait wait) {
+                                                    Sync sync) {
+  constexpr bool PF = MODE != kLoadDirect;
   const bool active = s_raw < p.S;
   const int s = active ? s_raw : 0;
   const size_t pair = (size_t)l * p.S + s;
@@ -139,12 +152,12 @@ __device__ __forceinline__ void route_group_streams(const RouteParams& p, const 
   sum_range = p.sum_range[pair];
 
   // The partial logits of the next token are requested before the current token is routed, so that their
-  // latency (L2, mostly) is off the critical path: up to kPartsMax parts of eight logits per lane in flight.
-  float4 raw[PF ? kPartsMax : 1][2];
+  // latency (L2, mostly) is off the critical path: up to NP parts of eight logits per lane in flight.
+  float4 raw[PF ? NP : 1][2];
   auto request = [&](int t) {
     const float* src = p.logits_in + (((size_t)t * p.L + l) * p.S + s) * E + e0;
 #pragma unroll
-    for (int q = 0; q < (PF ? kPartsMax : 1); ++q)
+    for (int q = 0; q < (PF ? NP : 1); ++q)
 #pragma unroll
       for (int h = 0; h < 2; ++h)
         if (q < p.n_partials && e0 + 4 * h < E) raw[q][h] = ldz4<COHERENT>((const float4*)(src + (size_t)q * p.partial_stride + 4 * h));
@@ -162,7 +175,7 @@ __device__ __forceinline__ void route_group_streams(const RouteParams& p, const 
         if (e0 + 4 * h < E) {
           v = raw[0][h];
 #pragma unroll
-          for (int q = 1; q < (PF ? kPartsMax : 1); ++q)
+          for (int q = 1; q < (PF ? NP : 1); ++q)
             if (q < p.n_partials) {
               const float4 u = raw[q][h];
               v.x = __fadd_rn(v.x, u.x), v.y = __fadd_rn(v.y, u.y), v.z = __fadd_rn(v.z, u.z), v.w = __fadd_rn(v.w, u.w);
@@ -170,7 +183,6 @@ __device__ __forceinline__ void route_group_streams(const RouteParams& p, const 
         }
         z[4 * h] = v.x, z[4 * h + 1] = v.y, z[4 * h + 2] = v.z, z[4 * h + 3] = v.w;
       }
-      if (t + 1 < p.n_steps) request(t + 1);
     } else if (vec4) {
 #pragma unroll
       for (int i = 0; i < kNE; i += 4) {
@@ -357,12 +369,25 @@ __device__ __forceinline__ void route_group_streams(const RouteParams& p, const 
     }
   };
 
-  if (PF) request(0);
-  for (int t = 0; t < p.n_steps; ++t) {
-    if (!wait(t)) break;
+  bool alive = true;
+  if (PF) {
+    alive = sync.wait(0);
+    if (alive) request(0);
+  }
+  for (int t = 0; t < p.n_steps && alive; ++t) {
+    if (!PF && !sync.wait(t)) break;
     Pre pre;
-    stage_a(t, pre);
+    stage_a(t, pre);            // with PF: consumes the registers that request(t) filled
+    bool requested = false;
+    if (PF && t + 1 < p.n_steps) {
+      requested = MODE == kPrefetchAll || sync.ready(t + 1);
+      if (requested) request(t + 1);
+    }
     stage_b(t, pre);
+    if (PF && t + 1 < p.n_steps && !requested) {
+      alive = sync.wait(t + 1);
+      if (alive) request(t + 1);
+    }
   }
 
   // ---- state back to memory ----------------------------------------------------------------------------------------------

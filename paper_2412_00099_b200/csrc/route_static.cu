@@ -18,7 +18,10 @@ constexpr int kMaxLayersForTotals = 1024;  // per-layer sums are staged in a hos
 // In host code this name is only a handle for cudaGetSymbolAddress; it is not a device pointer.
 static __device__ __align__(256) unsigned char g_route_scratch[kStaticScratchBytes];
 
-void* g_scratch_ptr[kMaxDevices];  // device address of the array, per device, resolved on first use
+// Device address of the array, per device ordinal, resolved on first use and kept for the life of the
+// process.  cudaDeviceReset unloads the library image from that device; the address cached here is then
+// stale, so a process that resets a device must not call this entry point on it again.
+void* g_scratch_ptr[kMaxDevices];
 
 size_t up256(size_t x) { return (x + 255) / 256 * 256; }
 
@@ -46,6 +49,11 @@ extern "C" int mcce_route_trace_static(const mcce_config* cfg, int32_t n_steps, 
   if (cfg->rerank_mode < MCCE_RERANK_CACHE_PRIOR || cfg->rerank_mode > MCCE_RERANK_CUMSUM) return MCCE_EINVAL;
   if (cfg->rerank_mode == MCCE_RERANK_MAX_RANK && (cfg->max_rank < 0 || cfg->max_rank > cfg->n_experts))
     return MCCE_EINVAL;
+  if (cfg->rerank_mode == MCCE_RERANK_CUMSUM && !(cfg->cum_threshold >= 0.f)) return MCCE_EINVAL;
+  // four-float accesses to the rows of logits (E a multiple of 4) and to the hidden rows
+  if (((uintptr_t)logits_in % ((cfg->n_experts & 3) ? 4 : 16)) || ((uintptr_t)hidden % 16)) return MCCE_EINVAL;
+  // refuse before any size is multiplied out: a state of L*S*E words must fit the array at all
+  if ((uint64_t)cfg->n_layers * (uint64_t)cfg->n_streams > kStaticScratchBytes / 4) return MCCE_ELIMIT;
 
   // layout of the state inside the static array; sizes beyond the array are refused
   const size_t LS = (size_t)cfg->n_layers * cfg->n_streams, E = cfg->n_experts, EW = (E + 31) / 32;
@@ -80,6 +88,7 @@ extern "C" int mcce_route_trace_static(const mcce_config* cfg, int32_t n_steps, 
   p.stamp = (uint32_t*)(base + o_stamp), p.ever = (uint32_t*)(base + o_ever);
   p.sum_range = (float*)(base + o_sum), p.miss = (uint32_t*)(base + o_miss), p.cold = (uint32_t*)(base + o_cold);
   p.sel_idx = sel_idx, p.sel_w = sel_w, p.logits_out = nullptr, p.tok0 = 0u, p.cnt0 = 0u;
+  p.err_nonfinite = nullptr;
   if (launch_route(p, st) != cudaSuccess) return MCCE_ECUDA;
 
   if (totals_host) {

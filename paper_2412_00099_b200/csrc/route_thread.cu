@@ -17,7 +17,8 @@ __global__ void __launch_bounds__(kThreads) route_group_kernel(const RouteParams
   const int blocks_per_layer = (p.S + kPerCta - 1) / kPerCta;
   const int l = blockIdx.x / blocks_per_layer;
   const int s_raw = (blockIdx.x % blocks_per_layer) * kPerCta + threadIdx.x / G;
-  rgroup::route_group_streams<G, KMAX, PF, false>(p, l, s_raw, threadIdx.x % G, [](int) { return true; });
+  rgroup::route_group_streams<G, KMAX, PF ? rgroup::kPrefetchAll : rgroup::kLoadDirect, kPartsMax, false>(
+      p, l, s_raw, threadIdx.x % G, rgroup::AllPresent());
 }
 
 template <int G, bool PF>

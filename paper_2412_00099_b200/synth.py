@@ -12,11 +12,17 @@ Generator definition (the CUDA generator kernels implement the same definition i
 * Normals: Box-Muller on two 24-bit uniforms, with ln, sin and cos evaluated by short series that
   use only +, -, *, / and sqrt in a fixed order and no fused multiply-add.  Every such operation is
   correctly rounded by IEEE-754, so the CPU (numpy float32) and the GPU produce identical bits.
+* `synth_host.c` is the same definition in plain C for the host (compiled on first use; the numpy code below is
+  the fallback and the reference it is tested against).
 * AR(1) hidden states: h_0 = n_0, h_t = rho*h_{t-1} + sqrt(1-rho^2)*n_t (fp32, mul, mul, add);
   emitted x_t = h_t + topic_offset, rounded to bf16 (ties to even) for the bf16 workloads.
 """
 from __future__ import annotations
 
+import ctypes
+import os
+import subprocess
+from concurrent.futures import ThreadPoolExecutor
 from dataclasses import dataclass, replace
 
 import numpy as np
@@ -101,18 +107,82 @@ def _box_muller(xa, xb):
 
 _CHUNK = 1 << 20     # elements per work item when a large draw is split over host threads
 
+# ---- the same definition compiled from synth_host.c (identical bits, much faster); numpy is the fallback ------
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_HOST_SRC = os.path.join(_HERE, "synth_host.c")
+_HOST_LIB = os.path.join(_HERE, "libsynth_host.so")
+_host = None
+
+
+def build_host(force: bool = False):
+    """Compiles synth_host.c with gcc (no fused multiply-add, no fast-math); returns the library path or None."""
+    try:
+        if force or not os.path.exists(_HOST_LIB) or os.path.getmtime(_HOST_LIB) < os.path.getmtime(_HOST_SRC):
+            subprocess.check_call(["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-ffp-contract=off", "-fno-fast-math",
+                                   "-o", _HOST_LIB, _HOST_SRC, "-lm"], stderr=subprocess.DEVNULL)
+        return _HOST_LIB
+    except (OSError, subprocess.CalledProcessError):
+        return None
+
+
+def _host_lib():
+    global _host
+    if _host is None:
+        path = None if os.environ.get("MCCE_SYNTH_NUMPY") else build_host()
+        _host = False
+        if path:
+            try:
+                lib = ctypes.CDLL(path)
+                lib.synth_fill.argtypes = [ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint64,
+                                           ctypes.c_uint64, ctypes.c_float, ctypes.c_int, ctypes.c_void_p]
+                lib.synth_fill.restype = None
+                lib.synth_hidden_step.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_uint64,
+                                                  ctypes.c_float, ctypes.c_float, ctypes.c_int, ctypes.c_int,
+                                                  ctypes.c_void_p]
+                lib.synth_hidden_step.restype = None
+                _host = lib
+            except OSError:
+                _host = False
+    return _host or None
+
+
+def _fill(seed, tensor_id, t, start, count, std, bf16):
+    """std * normals of elements [start, start+count), fp32 or bf16 bits, over all host threads."""
+    lib = _host_lib()
+    out = np.empty(count, np.uint16 if bf16 else np.float32)
+    if lib is None:
+        x = _normal_numpy(seed, tensor_id, t, start, count) * _F(std)
+        return to_bf16_bits(x) if bf16 else x
+    pieces = [(o, min(_CHUNK, count - o)) for o in range(0, count, _CHUNK)]
+
+    def fill(piece):
+        o, n = piece
+        lib.synth_fill(seed & 0xFFFFFFFF, tensor_id, t, start + o, n, float(_F(std)), int(bool(bf16)),
+                       out[o:o + n].ctypes.data)
+
+    if len(pieces) > 1:
+        with ThreadPoolExecutor(os.cpu_count() or 1) as ex:
+            list(ex.map(fill, pieces))
+    else:
+        for piece in pieces:
+            fill(piece)
+    return out
+
 
 def normal(seed: int, tensor_id: int, t: int, start: int, count: int) -> np.ndarray:
     """Standard normals for flat elements [start, start+count) of tensor `tensor_id` at step t (fp32)."""
+    return _fill(seed, tensor_id, t, start, count, 1.0, False)
+
+
+def _normal_numpy(seed: int, tensor_id: int, t: int, start: int, count: int) -> np.ndarray:
+    """The definition in numpy (what synth_host.c and the CUDA generator reproduce bit for bit)."""
     if count > 2 * _CHUNK and start % 4 == 0:
-        import os
-        from concurrent.futures import ThreadPoolExecutor
         out = np.empty(count, np.float32)
         pieces = [(o, min(_CHUNK, count - o)) for o in range(0, count, _CHUNK)]
 
         def fill(piece):
             o, n = piece
-            out[o:o + n] = normal(seed, tensor_id, t, start + o, n)
+            out[o:o + n] = _normal_numpy(seed, tensor_id, t, start + o, n)
 
         with ThreadPoolExecutor(os.cpu_count() or 1) as ex:
             list(ex.map(fill, pieces))
@@ -145,8 +215,8 @@ def bf16_bits_to_f32(b: np.ndarray) -> np.ndarray:
 
 
 def scaled_normal(seed, tensor_id, t, start, count, std: float, bf16: bool) -> np.ndarray:
-    x = normal(seed, tensor_id, t, start, count) * _F(std)
-    return to_bf16_bits(x) if bf16 else x
+    """std * n (one fp32 multiplication), as fp32 or as bf16 bit patterns."""
+    return _fill(seed, tensor_id, t, start, count, std, bf16)
 
 
 # ---------------------------------------------------------------------------------------------------
@@ -211,6 +281,32 @@ class Workload:
             return np.stack([normal(self.seed, tid, t, (l * S + s) * d, d) for l, s in rows])
 
         off = draw(T_OFFSET, 0) * _F(np.sqrt(0.5)) if self.topic_offset else None
+        lib = _host_lib()
+        if lib is not None:
+            # the same recurrence through synth_host.c, in place and over all host threads
+            h = None
+            for t in range(T):
+                n = np.ascontiguousarray(draw(T_NOISE, t))
+                if h is None:
+                    h = np.empty_like(n)
+                out = np.empty(n.shape, np.uint16 if self.bf16 else np.float32)
+                flat_h, flat_n, flat_o = h.reshape(-1), n.reshape(-1), out.reshape(-1)
+                flat_off = None if off is None else np.ascontiguousarray(off).reshape(-1)
+                pieces = [(o, min(_CHUNK, flat_n.size - o)) for o in range(0, flat_n.size, _CHUNK)]
+
+                def step(piece, t=t, flat_h=flat_h, flat_n=flat_n, flat_o=flat_o, flat_off=flat_off):
+                    o, m = piece
+                    lib.synth_hidden_step(flat_h[o:].ctypes.data, flat_n[o:].ctypes.data,
+                                          None if flat_off is None else flat_off[o:].ctypes.data, m, float(rho),
+                                          float(c), int(t == 0), int(self.bf16), flat_o[o:].ctypes.data)
+
+                if len(pieces) > 1:
+                    with ThreadPoolExecutor(os.cpu_count() or 1) as ex:
+                        list(ex.map(step, pieces))
+                else:
+                    step(pieces[0])
+                yield out
+            return
         h = None
         for t in range(T):
             n = draw(T_NOISE, t)

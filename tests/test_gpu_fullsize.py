@@ -2,10 +2,21 @@
 per token): the Qwen1.5-MoE-A2.7B-shaped workload (24 layers x 256 streams, 60+4 experts) that the bench line is
 quoted on, and the OLMoE-, DeepSeek-V2-Lite- and Mixtral-8x7B-shaped ones.
 
-The library's inputs are generated on the device; the oracle's inputs for the sampled (layer, stream)
-pairs are regenerated on the host from the same seeded definition (the two generators agree bit for bit,
-which is re-checked here on the sampled expert matrices).  Sampled outputs are compared one by one; the
-rest is checked through properties that hold at any size."""
+The library's inputs are generated on the device; every oracle input is regenerated on the host from the same
+seeded definition and compared with the device's bits where both exist.  Three levels of comparison:
+  * every (layer, stream) pair, every token: the oracle, advanced on the logits the library reports, must
+    reproduce selection, weights, cache state and counters exactly;
+  * six sampled pairs: additionally the library's logits against the oracle's own fp64 logits from
+    host-generated hidden rows, with near-tie accounting where the oracle's own decision differs;
+  * the expert FFN output y of at least 32 (layer, stream) pairs on each of the last three tokens, recomputed by
+    the oracle from host-generated hidden rows and expert matrices, element by element within the FFN tolerance.
+    The pairs cover every layer (for the Mixtral-shaped workload, whose experts have 176 M parameters each, four
+    layers spread over the depth); inside a layer they are picked so that few distinct expert matrices have to
+    be regenerated on the host.
+The rest is checked through properties that hold at any size."""
+import os
+from concurrent.futures import ThreadPoolExecutor
+
 import numpy as np
 import pytest
 import torch
@@ -14,22 +25,31 @@ from paper_2412_00099_b200 import synth
 
 pytestmark = pytest.mark.gpu
 
+FFN_TOKENS = 3      # the last tokens of a case get their FFN outputs recomputed
+FFN_PAIRS = 32      # at least this many (layer, stream) pairs on each of them
+
+
 def sample_pairs(wl):
     """Six (layer, stream) pairs spread over the workload, corners included."""
     L, S = wl.L, wl.S
     return [(0, 0), (L // 8, S // 15), (L // 2, S // 2), (L - 1, S - 1), (L // 3, S // 4), (2 * L // 3, 4 * S // 5)]
 
 
-# workload, tokens, pairs whose FFN output is recomputed on the host (their expert matrices are regenerated there)
-CASES = [(synth.QWEN, 5, 4), (synth.OLMOE, 3, 2), (synth.DEEPSEEK, 3, 2), (synth.MIXTRAL, 3, 1)]
+def ffn_layers(wl):
+    if 3 * wl.d * wl.I > 50_000_000:                    # very large experts: four layers over the depth
+        return [0, wl.L // 3, 2 * wl.L // 3, wl.L - 1]
+    return list(range(wl.L))
+
+
+CASES = [(synth.QWEN, 5), (synth.OLMOE, 4), (synth.DEEPSEEK, 4), (synth.MIXTRAL, 4)]
 
 
 def bits(t: torch.Tensor) -> np.ndarray:
     return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
 
 
-@pytest.mark.parametrize("wl,T_STEPS,FFN_SAMPLES", CASES, ids=[c[0].name for c in CASES])
-def test_full_size_sampled_parity(wl, T_STEPS, FFN_SAMPLES):
+@pytest.mark.parametrize("wl,T_STEPS", CASES, ids=[c[0].name for c in CASES])
+def test_full_size_parity(wl, T_STEPS):
     from oracle import oracle as orc
     from paper_2412_00099_b200 import binding as mb
     import helpers as H
@@ -38,6 +58,7 @@ def test_full_size_sampled_parity(wl, T_STEPS, FFN_SAMPLES):
     torch.cuda.empty_cache()            # the previous case's weights (tens of GB) must be gone first
     dev = torch.device("cuda")
     bf = torch.bfloat16
+    threads = os.cpu_count() or 1
     eng = mb.engine_for(wl)
     assert eng.uses_tensor_path()
     Wr = mb.gen_normal(torch.empty((wl.L, wl.E, wl.d), dtype=torch.float32, device=dev), wl.seed, synth.T_ROUTER,
@@ -50,17 +71,33 @@ def test_full_size_sampled_parity(wl, T_STEPS, FFN_SAMPLES):
               if (wl.n_shared or not k.startswith("sh")) else None) for k, (tid, shp) in W.items()}
     eng.set_router(Wr)
     eng.set_experts(**Wt)
-    assert np.array_equal(Wr.cpu().numpy(), wl.router())          # router: device generator == host generator
+    Wr_host = wl.router()
+    assert np.array_equal(Wr.cpu().numpy(), Wr_host)               # router: device generator == host generator
 
-    # the oracle follows the sampled pairs only: one "layer" per sample, one stream each
+    # oracle A follows every pair on the library's logits; oracle B follows the sampled pairs on its own logits
+    o_all = orc.Oracle(orc.OracleConfig(wl.L, wl.E, wl.K, wl.J, wl.n_shared, wl.d, wl.I, wl.C, wl.S, wl.lam, 0, 1, 1),
+                       threads=threads)
     n = len(SAMPLES)
-    Wr_s = np.ascontiguousarray(wl.router()[[l for l, _ in SAMPLES]])
+    Wr_s = np.ascontiguousarray(Wr_host[[l for l, _ in SAMPLES]])
     o = orc.Oracle(orc.OracleConfig(n, wl.E, wl.K, wl.J, wl.n_shared, wl.d, wl.I, wl.C, 1, wl.lam, 0, 1, 1))
     host_x = wl.hidden_trace(T_STEPS, rows=SAMPLES)
 
+    mats = {}                                                       # (tensor id, layer, expert) -> host matrix
+
+    def expert(shared, l, e):
+        ids = (synth.T_SH_WG, synth.T_SH_WU, synth.T_SH_WD) if shared else (synth.T_WG, synth.T_WU, synth.T_WD)
+        out = []
+        for tid in ids:
+            if (tid, l, e) not in mats:
+                mats[(tid, l, e)] = wl.expert_matrix(tid, l, e)
+            out.append(mats[(tid, l, e)])
+        return out
+
     state = torch.empty(wl.L * wl.S * wl.d, dtype=torch.float32, device=dev)
     x = torch.empty((wl.L, wl.S, wl.d), dtype=bf, device=dev)
-    near = 0
+    near, ffn_checked, worst_ffn = 0, 0, 0.0
+    layers = ffn_layers(wl)
+    per_layer = -(-FFN_PAIRS // len(layers))
     for t in range(T_STEPS):
         mb.gen_hidden_step(state, x, wl.seed, t, wl.rho, wl.topic_offset)
         sel, w, z = eng.route_step(hidden=x, want_logits=True)
@@ -80,7 +117,12 @@ def test_full_size_sampled_parity(wl, T_STEPS, FFN_SAMPLES):
             assert np.array_equal(offsets[l], np.concatenate([[0], np.cumsum(np.bincount(flat, minlength=wl.E))]))
             assert np.array_equal(perm[l], np.argsort(flat, kind="stable"))
 
-        # ---- sampled pairs against the oracle --------------------------------------------------------
+        # ---- every pair: the recurrence on the library's logits ----------------------------------------
+        osel_all, ow_all = o_all.route(z_h)
+        assert np.array_equal(sel_h, osel_all), "selection differs at token %d" % t
+        assert np.allclose(w_h, ow_all, rtol=1e-5, atol=1e-7)
+
+        # ---- sampled pairs: the library's logits against the oracle's own ------------------------------
         xs = next(host_x)                                              # [n, d] bf16 bits from the host generator
         for i, (l, s) in enumerate(SAMPLES):
             assert np.array_equal(bits(x[l, s]), xs[i])                # same inputs on both sides
@@ -93,35 +135,64 @@ def test_full_size_sampled_parity(wl, T_STEPS, FFN_SAMPLES):
         osel, ow = o.route(z_g)
         for i, (l, s) in enumerate(SAMPLES):
             assert np.array_equal(sel_h[l, s], osel[i, 0])
-            assert np.allclose(w_h[l, s], ow[i, 0], rtol=1e-5, atol=1e-7)
             if not np.array_equal(sel_own[i, 0], osel[i, 0]):
                 assert margin[i, 0] < H.NEAR_TIE
                 near += 1
 
-        if t == T_STEPS - 1:                                           # FFN outputs of a few pairs, recomputed
-            for i, (l, s) in enumerate(SAMPLES[:FFN_SAMPLES]):
+        # ---- FFN outputs of >= 32 pairs, recomputed from host-generated inputs ---------------------------
+        if t >= T_STEPS - FFN_TOKENS:
+            chosen = []
+            for l in layers:
+                have = {e for (tid, ll, e) in mats if ll == l and tid == synth.T_WG}
+                start = (37 * l + 11) % wl.S                            # a different first stream per layer
+                for _ in range(per_layer):
+                    order = [(start + i) % wl.S for i in range(wl.S)]
+                    cost = lambda s: sum(int(e) not in have for e in osel_all[l, s])
+                    s = min((s for s in order if (l, s) not in chosen), key=cost)
+                    chosen.append((l, s))
+                    have |= {int(e) for e in osel_all[l, s]}
+            # hidden rows of the chosen pairs at token t, from the host definition of the trace
+            rows = list(wl.hidden_trace(t + 1, rows=chosen))[-1]
+            first_of_layer = {}
+            for i, (l, s) in enumerate(chosen):
+                assert np.array_equal(bits(x[l, s]), rows[i])
+                first_of_layer.setdefault(l, i)
+
+            def ref_of(i):
+                l, s = chosen[i]
                 acc = np.zeros(wl.d, np.float64)
                 for k in range(wl.K):
-                    e = int(osel[i, 0, k])
-                    mats = [wl.expert_matrix(tid, l, e) for tid in (synth.T_WG, synth.T_WU, synth.T_WD)]
-                    if k == 0:                                         # device weights == host weights
-                        assert np.array_equal(bits(Wt["Wg"][l, e]), mats[0])
-                        assert np.array_equal(bits(Wt["Wd"][l, e]), mats[2])
-                    acc += float(ow[i, 0, k]) * orc.expert_ffn(xs[i], *mats, 1)
+                    acc += float(ow_all[l, s, k]) * orc.expert_ffn(rows[i], *expert(False, l, int(osel_all[l, s, k])), 1)
                 for q in range(wl.n_shared):
-                    mats = [wl.expert_matrix(tid, l, q) for tid in (synth.T_SH_WG, synth.T_SH_WU, synth.T_SH_WD)]
-                    acc += orc.expert_ffn(xs[i], *mats, 1)
-                err = H.ffn_close(y_h[l, s], acc.astype(np.float32))
-                print("full-size FFN sample (l=%d, s=%d): max abs err %.2e" % (l, s, err[0]))
+                    acc += orc.expert_ffn(rows[i], *expert(True, l, q), 1)
+                return acc.astype(np.float32)
 
-    # cache state and counters of the sampled pairs
-    order, ever, dsum, cnt = eng.cache_state()
-    o_order = o.order()
-    for i, (l, s) in enumerate(SAMPLES):
-        assert np.array_equal(order[l, s], o_order[i, 0])
-        assert np.array_equal(ever[l, s], o.ever[i, 0])
-        assert dsum[l, s].view(np.uint32) == o.sum_range[i, 0].view(np.uint32)
-    total, per_layer = eng.cache_stats()
+            for l in layers:                                            # generate serially (the generator is threaded)
+                for i, (ll, s) in enumerate(chosen):
+                    if ll == l:
+                        for k in range(wl.K):
+                            expert(False, l, int(osel_all[l, s, k]))
+                        for q in range(wl.n_shared):
+                            expert(True, l, q)
+                i0 = first_of_layer[l]                                  # device weights == host weights
+                e0 = int(osel_all[l, chosen[i0][1], 0])
+                assert np.array_equal(bits(Wt["Wg"][l, e0]), mats[(synth.T_WG, l, e0)])
+                assert np.array_equal(bits(Wt["Wd"][l, e0]), mats[(synth.T_WD, l, e0)])
+            with ThreadPoolExecutor(threads) as ex:
+                refs = list(ex.map(ref_of, range(len(chosen))))
+            for i, (l, s) in enumerate(chosen):
+                err = H.ffn_close(y_h[l, s], refs[i])
+                worst_ffn = max(worst_ffn, err[0])
+            ffn_checked += len(chosen)
+            assert len(chosen) >= FFN_PAIRS
+
+    # cache state and counters: every pair
+    H.assert_state_equal(eng, o_all)
+    total, per_layer_stats = eng.cache_stats()
     assert total[0] == T_STEPS * wl.L * wl.S and total[1] == total[0] * wl.K
     assert 0 < total[3] <= total[2] <= total[1]
-    print("full size: %d sampled steps, %d near ties, miss rate %.3f" % (T_STEPS * n, near, total[2] / total[1]))
+    print("full size %s: %d tokens of all %d pairs identical; %d sampled steps with %d near ties; %d FFN outputs "
+          "recomputed over %d layers (%d host expert matrices), max abs err %.2e; miss rate %.3f"
+          % (wl.name, T_STEPS, wl.L * wl.S, T_STEPS * n, near, ffn_checked, len(layers), len(mats), worst_ffn,
+             total[2] / total[1]))
+    eng.close()

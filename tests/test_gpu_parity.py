@@ -470,6 +470,41 @@ def test_pipelined_host_steps_match_synchronous_ones():
     assert a.cache_stats()[0] == b.cache_stats()[0]
 
 
+@pytest.mark.parametrize("deterministic", [False, True])
+def test_pipelined_device_steps_match_step_by_step_calls(deterministic):
+    """mcce_pipeline_submit (routing + grouping of step t+1 on an internal stream while the experts of step t run)
+    against one mcce_route_step + mcce_moe_forward per token: same selections, cache state and counters; y bit
+    for bit in deterministic mode, else equal up to the order of the atomic adds."""
+    wl = synth.QWEN.with_(L=3, S=40, E=16, K=4, C=8, d=256, I=384, n_shared=1)
+    Wr, W = wl.router(), H.weights_for(wl)
+    a, b = mb.engine_for(wl, deterministic=deterministic), mb.engine_for(wl, deterministic=deterministic)
+    for e in (a, b):
+        e.set_router(H.to_dev(Wr))
+        e.set_experts(**{k: (None if v is None else H.to_dev(v)) for k, v in W.items()})
+    T = 9
+    xs = torch.stack([H.to_dev(x) for x in wl.hidden_trace(T)])
+    torch.cuda.synchronize()
+    ys = torch.zeros((T, wl.L, wl.S, wl.d), dtype=torch.float32, device="cuda")
+    sels = torch.zeros((T, wl.L, wl.S, wl.K), dtype=torch.int32, device="cuda")
+    for t in range(T):
+        b.pipeline_submit(xs[t], ys[t], sels[t])
+    b.pipeline_wait()
+    for t in range(T):
+        sel, w = a.route_step(hidden=xs[t:t + 1])
+        y = a.moe_forward(xs[t], sel[0], w[0])
+        assert torch.equal(sel[0], sels[t]), "token %d" % t
+        if deterministic:
+            assert torch.equal(y, ys[t])
+        else:
+            assert torch.allclose(y, ys[t], rtol=1e-5, atol=1e-6)
+    assert a.cache_stats()[0] == b.cache_stats()[0]
+    assert np.array_equal(a.cache_state()[0], b.cache_state()[0])
+    # the context goes on with the ordinary calls afterwards
+    sel_a, _ = a.route_step(hidden=xs[:1])
+    sel_b, _ = b.route_step(hidden=xs[:1])
+    assert torch.equal(sel_a, sel_b)
+
+
 # ---- argument checking: errors come back as codes, nothing is launched ------------------------------------
 def test_bad_arguments_are_rejected():
     with pytest.raises(mb.McceError):

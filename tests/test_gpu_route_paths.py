@@ -93,7 +93,7 @@ FUSED_CASES = [
     (synth.QWEN, dict(L=20, S=200, d=512, C=15), 8),
     (synth.OLMOE, dict(L=19, S=130, d=512), 5),
     (synth.MIXTRAL, dict(L=32, S=64, d=1024), 8),
-    (synth.QWEN, dict(L=24, S=97, d=448, E=37, K=3, C=9), 4),     # experts not a multiple of 4, one ragged tile
+    (synth.QWEN, dict(L=24, S=97, d=448, E=36, K=3, C=9), 4),     # experts not a multiple of 8, one ragged tile
 ]
 
 
@@ -116,6 +116,7 @@ def test_fused_route_kernel_from_hidden_states(base, kw, chunk):
     (synth.QWEN, dict(L=3, S=300, d=512, C=30)),        # three stream tiles, the last one ragged
     (synth.DEEPSEEK, dict(L=2, S=128, d=2048)),
     (synth.QWEN, dict(L=2, S=40, d=256, E=80, K=4)),    # the most experts the router-resident GEMM takes
+    (synth.QWEN, dict(L=24, S=97, d=448, E=37, K=3, C=9)),   # experts not a multiple of 4: no fused kernel either
 ])
 def test_router_resident_gemm_then_tail(base, kw):
     wl = base.with_(**kw)
@@ -123,7 +124,7 @@ def test_router_resident_gemm_then_tail(base, kw):
     xs = np.stack(list(wl.hidden_trace(10)))
     eng, o = mb.engine_for(wl, ffn_impl=mb.FFN_SIMT, route_impl=mb.ROUTE_FUSED), H.oracle_for(wl)
     eng.set_router(H.to_dev(Wr))
-    assert eng.router_kernel_kind(8) == mb.ROUTER_RESIDENT_TAIL     # too few layers for the fused kernel, even if asked
+    assert eng.router_kernel_kind(8) == mb.ROUTER_RESIDENT_TAIL     # no fused kernel for this shape, even if asked
     near, dz = follow_chunked(eng, o, Wr, xs[:8], 8, mb.ROUTER_RESIDENT_TAIL)
     near2, dz2 = follow_chunked(eng, o, Wr, xs[8:], 1, mb.ROUTER_RESIDENT_TAIL)
     print("%s resident: %d near ties, max logit err %.2e" % (wl.name, near + near2, max(dz, dz2)))

@@ -40,3 +40,29 @@ def test_weights_have_the_stated_spread():
     assert abs(w.std() - 0.02) < 2e-4 and abs(w.mean()) < 2e-4
     r = synth.TINY.router()
     assert abs(r.var() - 1.0 / synth.TINY.d) < 0.15 / synth.TINY.d * 8               # N(0, 1/d), 512 samples
+
+
+def test_compiled_host_generator_equals_the_numpy_definition(monkeypatch):
+    """synth_host.c against the numpy code it restates: normals (ragged starts, beyond 2^32 blocks), scaled bf16
+    weights and the AR(1) trace, bit for bit."""
+    assert synth.build_host() is not None, "gcc could not build synth_host.c"
+    synth._host = None
+    cases = [(1, 2, 0, 0, 1000), (5, 3, 7, 4096 + 3, 100_003), (9, 8, 13, (1 << 34) + 8, 5000), (0, 11, 2, 1, 7),
+             (3, 8, 1, 0, 2_500_000)]
+    fast = [(synth.normal(*c), synth.scaled_normal(*c, 0.02, True)) for c in cases]
+    wls = (synth.TINY.with_(S=5, L=2), synth.QWEN.with_(L=2, S=7, d=64), synth.MIXTRAL.with_(L=1, S=3, d=128))
+    fast_traces = [list(w.hidden_trace(5)) + list(w.hidden_trace(5, rows=[(0, 1), (w.L - 1, 2)])) for w in wls]
+    assert synth._host_lib() is not None
+    monkeypatch.setenv("MCCE_SYNTH_NUMPY", "1")
+    synth._host = None
+    try:
+        assert synth._host_lib() is None
+        for c, (n, b) in zip(cases, fast):
+            assert np.array_equal(n.view(np.uint32), synth.normal(*c).view(np.uint32))
+            assert np.array_equal(b, synth.scaled_normal(*c, 0.02, True))
+        for w, tr in zip(wls, fast_traces):
+            slow = list(w.hidden_trace(5)) + list(w.hidden_trace(5, rows=[(0, 1), (w.L - 1, 2)]))
+            for a, b in zip(tr, slow):
+                assert a.dtype == b.dtype and a.shape == b.shape and np.array_equal(a.view(np.uint8), b.view(np.uint8))
+    finally:
+        synth._host = None
