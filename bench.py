@@ -92,6 +92,9 @@ def parse_args():
     ap.add_argument("--ffn", default="auto", choices=["auto", "simt", "tensor"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--deterministic", action="store_true",
+                    help="slot-order combine on the tensor-core path (bit-identical repeats) instead of atomic adds")
+    ap.add_argument("--checked", action="store_true", help="checked mode of the context (consistency kernels after each pass)")
     ap.add_argument("--step-by-step", action="store_true",
                     help="one mcce_route_step + mcce_moe_forward per token on one stream instead of mcce_pipeline_submit")
     ap.add_argument("--no-steady-state", action="store_true",
@@ -336,7 +339,8 @@ def main_arm(args):
     rerank = {"prior": mb.RERANK_CACHE_PRIOR, "maxrank": mb.RERANK_MAX_RANK, "cumsum": mb.RERANK_CUMSUM}[args.rerank]
     max_rank = min(wl.E, args.max_rank if args.max_rank is not None else 2 * wl.K)
     eng = mb.engine_for(wl, ffn_impl=ffn_impl, device=local, rerank_mode=rerank, max_rank=max_rank,
-                        cum_threshold=args.cum_p, track_lifetime=args.lifetimes)
+                        cum_threshold=args.cum_p, track_lifetime=args.lifetimes, deterministic=args.deterministic,
+                        checked=args.checked)
     wdt = torch.bfloat16 if wl.bf16 else torch.float32
 
     # ---- weights, generated on the device ------------------------------------------------------------
@@ -490,6 +494,7 @@ def main_arm(args):
             "config": config_of(wl, {"l2": "inputs larger than L2: %.1f GB of expert weights streamed per step"
                                            % ((bytes_up + bytes_down) / 1e9),
                                      "ffn_path": "tensor" if _uses_tensor(eng) else "simt",
+                                     "combine": "slot order (deterministic)" if args.deterministic else "default",
                                      "layer_mode": "chained through a residual stream" if args.chained else "independent",
                                      "call": ("mcce_decode_step_chained" if args.chained else
                                               "mcce_route_step + mcce_moe_forward per token" if args.step_by_step else

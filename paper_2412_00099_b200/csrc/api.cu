@@ -12,11 +12,11 @@
 using namespace mcce;
 
 constexpr int kMaxPairs = 1024;
-// When MCCE_ROUTE_AUTO takes the single fused kernel: from four tokens per launch (for fewer the two launches
-// are faster) and with at most 16 experts (with more, the tail inside the fused kernel -- 80 registers, no
-// prefetch of the next token's logits -- is a slower chain than the stand-alone tail; measured on the
-// Mixtral-shaped workload 60 against 86 us for eight tokens, on the OLMoE-shaped one 180 against 156).
-constexpr int kFusedMinTokens = 4, kFusedMaxExperts = 16;
+// When MCCE_ROUTE_AUTO takes the single fused kernel: from four tokens per launch (for fewer the two launches are
+// faster) and while a CTA of it runs at most 12 tail warps.  With more, a thread has 80 registers, the tail
+// spills and becomes the slower chain.  Measured, eight tokens per launch, fused against two kernels:
+// Qwen-shaped (11 tail warps) 90 against 97 us, Mixtral-shaped (1) 60 against 85, OLMoE-shaped (16) 203 against 163.
+constexpr int kFusedMinTokens = 4, kFusedMaxTailWarps = 12;
 
 struct mcce_ctx {
   mcce_config cfg;
@@ -148,9 +148,8 @@ Layout layout_of(const mcce_config& c) {
   o.st_y2 = take(L * S * d * 4);
   const bool rg = router_gemm_applicable(c);
   o.wr_terms = take(rg ? 3 * L * E * d * 2 : 0);
-  // logits of up to router_gemm_steps_max() tokens; the router-resident kernels write one array per K part, the
-  // fused one a further array with their sum
-  const size_t z_slots = (size_t)router_gemm_steps_max() * (router_gemm_res_applicable(c) ? router_gemm_res_parts_max() + 1 : 1);
+  // logits of up to router_gemm_steps_max() tokens; the router-resident kernels write one array per K part
+  const size_t z_slots = (size_t)router_gemm_steps_max() * (router_gemm_res_applicable(c) ? router_gemm_res_parts_max() : 1);
   o.z_buf = take(rg ? z_slots * L * S * E * 4 : 0);
   o.z_ready = take(rg ? route_fused_counter_words((int)L, router_gemm_steps_max(), (int)S) * 4 : 0);   // counters of the fused kernel
   o.load_tok = take(c.track_lifetime ? L * S * E * 4 : 0);
@@ -162,7 +161,7 @@ Layout layout_of(const mcce_config& c) {
 bool use_fused(const mcce_ctx* ctx, int n_tokens) {
   if (!ctx->rg.fused_ready || ctx->cfg.route_impl == MCCE_ROUTE_TWO_KERNELS) return false;
   if (ctx->cfg.route_impl == MCCE_ROUTE_FUSED) return true;
-  return n_tokens >= kFusedMinTokens && ctx->cfg.n_experts <= kFusedMaxExperts;
+  return n_tokens >= kFusedMinTokens && ctx->rg.fused_tail_warps <= kFusedMaxTailWarps;
 }
 
 int cuda_fail(mcce_ctx* ctx, cudaError_t e) {

@@ -92,6 +92,7 @@ struct RouterGemmPlan {
   int res_ready, res_parts;   // K parts (= partial logit arrays) of the router-resident kernel
   int res_parts_single;       // the same for a launch of one layer at a time
   int fused_ready, fused_parts;   // the same for the kernel that also runs the routing tail (route_fused.cu)
+  int fused_tail_warps;           // tail warps per CTA of that kernel
 };
 bool router_gemm_applicable(const mcce_config& c);
 int router_gemm_steps_max();

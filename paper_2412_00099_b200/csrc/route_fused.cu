@@ -4,17 +4,18 @@
 // next ones instead of following it in a second launch.
 //
 // A layer belongs to KS CTAs (one K part of the reduction each).  Warps 0-5 of a CTA are the GEMM (TMA
-// producer, MMA issuer, four epilogue warps).  An epilogue warp stores the partial logits of its K part for its
-// 32 rows of the (token, stream tile) and counts itself in on a counter of that (tile, row quadrant).  Two more
-// warps add the K parts up, in the fixed order 0 .. KS-1: for every tile and quadrant they wait (bounded) until
-// all KS parts have counted in, sum their CTA's share of the quadrant (a KS-th of its float4s, read back through
-// L2), store the summed logits and count in on the tile's "sum ready" counter.  The remaining warps of every CTA
-// are the tail: the S streams of the layer are dealt out to its KS CTAs, a group of lanes per stream as in
-// route_group.cuh; before a token they wait (bounded) for the sum-ready counters of the tiles they read, and they
-// ask for the next token's summed logits while they route the current one whenever those are ready by then.
-// The launch is cooperative, so every CTA that a warp waits for is resident; the GEMM warps wait for nothing
-// outside their CTA, the summing warps only for GEMM warps, the tail only for summing warps, so the waits cannot
-// form a cycle.
+// producer, MMA issuer, four epilogue warps); an epilogue warp stores the partial logits of its K part for its
+// 32 rows of the (token, stream tile) and then counts itself in on the tile's counter, after a device-wide
+// fence.  The remaining warps are the tail: the S streams of the layer are dealt out to its KS CTAs, a group of
+// lanes per stream as in route_group.cuh.  Before a token they wait (bounded) until all 4 x KS epilogue warps of
+// the layer have counted in on the tiles they read, then read the KS partial sums (L2-coherent loads) and add
+// them in the fixed order 0 .. KS-1.  The launch is cooperative, so every CTA that a tail warp waits for is
+// resident; the GEMM warps wait for nothing outside their CTA, so the waits cannot form a cycle.
+//
+// Measured alternatives (Qwen-shaped, eight tokens per launch, this form: 90 us): holding the next token's KS
+// parts in registers while the current token is routed (64 more registers than the 96 a thread has here: spills,
+// 120 us); two more warps per CTA that add the parts up ahead of the tail, so that it reads one array (each
+// tile then passes through three more L2 round trips on two latency-bound warps: 164 us).
 #include "route_gemm_res.cuh"
 #include "route_group.cuh"
 
@@ -25,18 +26,16 @@ using namespace rres;
 namespace {
 
 constexpr int kGemmWarps = 6;      // TMA producer, MMA issuer, four epilogue warps
-constexpr int kSumWarps = 2;       // add up the K parts of finished tiles
-constexpr int kFrontWarps = kGemmWarps + kSumWarps;
+constexpr int kFrontWarps = kGemmWarps;
 constexpr int kMaxTailWarps = 16;
 
 struct FusedArgs {
   Geometry g;
   int Sc;               // streams of the layer routed by each of its CTAs
   int tail_warps;
-  float* Z;             // [KS][n_steps, L, S, E] partial logits, then one more such array: their sum
+  float* Z;             // [KS][n_steps, L, S, E] partial logits
   size_t z_stride;
-  uint32_t* part_ready; // [L][n_steps * n_tiles][4] K parts that have stored a row quadrant of a tile
-  uint32_t* sum_ready;  // [L][n_steps * n_tiles]    (row quadrant, CTA) shares of a tile that have been summed
+  uint32_t* part_ready; // [L][n_steps * n_tiles] epilogue warps (4 per K part) that have stored their rows of a tile
   uint32_t* err;
 };
 
@@ -71,11 +70,11 @@ __device__ __forceinline__ bool wait_count(const uint32_t* q, uint32_t target, v
   }
 }
 
-// What the tail asks before it reads the summed logits of a token: the sum-ready counters of the (at most two
-// distinct ends of the range of) stream tiles that the calling warp's streams lie in.
+// What the tail asks before it reads the partial logits of a token: the counters of the stream tiles that the
+// calling warp's streams lie in.
 struct TailSync {
-  const uint32_t* ready_l;   // sum_ready of this layer
-  uint32_t target;           // counts of a finished tile: 4 row quadrants x KS shares
+  const uint32_t* ready_l;   // part_ready of this layer
+  uint32_t target;           // counts of a finished tile: 4 epilogue warps x KS parts
   int n_tiles, tile_lo, tile_hi;
   volatile uint32_t* abort_flag;
   uint32_t* err;
@@ -122,47 +121,10 @@ route_fused_kernel(const __grid_constant__ Maps maps, const FusedArgs args, cons
       const size_t grow = (size_t)(t * a.L + l) * a.S + tile * kTileM + row;
       const bool row_ok = tile * kTileM + row < a.S;
       if (!drain_pair(a, m, tmem_base, kp, (uint32_t)i, quad, lane, Zp + grow * a.E, row_ok, args.err, 35u)) break;
-      uint32_t* cnt = args.part_ready + ((size_t)l * n_pairs + i) * 4 + quad;
+      uint32_t* cnt = args.part_ready + (size_t)l * n_pairs + i;
       __threadfence();   // this lane's part of the tile is visible device-wide before the warp counts in
       __syncwarp();
       if (lane == 0) atomicAdd(cnt, 1u);
-    }
-  } else if (warp < kFrontWarps) {
-    // ---- the K parts of every tile are added up, each CTA of the layer taking an equal share ------------------
-    // The 32 rows of a quadrant are one contiguous block of 32 * E floats in every part; CTA ks sums the float4s
-    // ks*32 + lane, then (ks + KS)*32 + lane, ... of that block (coalesced), parts in the order 0 .. KS-1.  This
-    // warp serves two of the four row quadrants.
-    float* Zsum = args.Z + (size_t)a.KS * args.z_stride;
-    const size_t stride4 = args.z_stride / 4;
-    bool alive = true;
-    for (int i = 0; i < n_pairs && alive; ++i) {
-      const int t = i / a.n_tiles, tile = i % a.n_tiles;
-      for (int quad = 2 * (warp - kGemmWarps); quad < 2 * (warp - kGemmWarps) + 2 && alive; ++quad) {
-        alive = wait_count(args.part_ready + ((size_t)l * n_pairs + i) * 4 + quad, (uint32_t)a.KS, m.abort_flag, args.err, 37u);
-        if (!alive) break;
-        const int rows_valid = min(32, max(0, a.S - tile * kTileM - quad * 32));
-        const int n4 = rows_valid * a.E / 4;
-        const size_t blk = ((size_t)(t * a.L + l) * a.S + tile * kTileM + quad * 32) * a.E;
-        const float4* src = (const float4*)(args.Z + blk);
-        float4* dst = (float4*)(Zsum + blk);
-#pragma unroll 2
-        for (int k = ks * 32 + lane; k < n4; k += 32 * a.KS) {
-          float4 u[kPartsMax];
-#pragma unroll
-          for (int q = 0; q < kPartsMax; ++q)
-            if (q < a.KS) u[q] = __ldcg(src + (size_t)q * stride4 + k);
-          float4 v = u[0];
-#pragma unroll
-          for (int q = 1; q < kPartsMax; ++q)
-            if (q < a.KS)
-              v.x = __fadd_rn(v.x, u[q].x), v.y = __fadd_rn(v.y, u[q].y), v.z = __fadd_rn(v.z, u[q].z),
-              v.w = __fadd_rn(v.w, u[q].w);
-          dst[k] = v;
-        }
-        __threadfence();
-        __syncwarp();
-        if (lane == 0) atomicAdd(args.sum_ready + (size_t)l * n_pairs + i, 1u);
-      }
     }
   } else {
     // ---- routing tail of this CTA's share of the layer's streams -------------------------------------------
@@ -171,11 +133,11 @@ route_fused_kernel(const __grid_constant__ Maps maps, const FusedArgs args, cons
     const int s_raw = idx < args.Sc ? ks * args.Sc + idx : a.S;   // past the share: idle group
     if (tw < args.tail_warps && ks * args.Sc + (tw * 32) / G < a.S) {
       TailSync sync;
-      sync.ready_l = args.sum_ready + (size_t)l * n_pairs, sync.n_tiles = a.n_tiles, sync.target = 4u * (uint32_t)a.KS;
+      sync.ready_l = args.part_ready + (size_t)l * n_pairs, sync.n_tiles = a.n_tiles, sync.target = 4u * (uint32_t)a.KS;
       sync.tile_lo = min(a.S - 1, ks * args.Sc + (tw * 32) / G) / kTileM;
       sync.tile_hi = min(a.S - 1, ks * args.Sc + min(args.Sc - 1, (tw * 32 + 31) / G)) / kTileM;
       sync.abort_flag = m.abort_flag, sync.err = args.err;
-      rgroup::route_group_streams<G, KMAX, rgroup::kPrefetchReady, 1, true>(p, l, s_raw, lane % G, sync);
+      rgroup::route_group_streams<G, KMAX, rgroup::kLoadDirect, 1, true>(p, l, s_raw, lane % G, sync);
     }
   }
   teardown(m, tmem_base, warp, 1);
@@ -242,9 +204,9 @@ cudaError_t launch_any(int G, int K, int TW, const Maps& m, const FusedArgs& a, 
 
 }  // namespace
 
-// Counters the kernel needs per launch: four part-ready and one sum-ready word per (layer, token, stream tile).
+// Counters the kernel needs per launch: one word per (layer, token, stream tile).
 size_t route_fused_counter_words(int n_layers, int n_steps, int n_streams) {
-  return (size_t)n_layers * n_steps * ((n_streams + kTileM - 1) / kTileM) * 5;
+  return (size_t)n_layers * n_steps * ((n_streams + kTileM - 1) / kTileM);
 }
 
 // Fixes the K-split of the fused kernel for this configuration, or leaves plan->fused_ready at 0 when the two-kernel
@@ -276,12 +238,13 @@ int route_fused_plan(const mcce_config& c, RouterGemmPlan* plan) {
   }
   if (best_ks == 0 || 2 * best_ctas < sms) return MCCE_OK;
   plan->fused_parts = best_ks;
+  plan->fused_tail_warps = ((c.n_streams + best_ks - 1) / best_ks * G + 31) / 32;
   plan->fused_ready = 1;
   return MCCE_OK;
 }
 
 // The routing step of n_steps tokens of all layers.  p carries the routing parameters and outputs; its logits
-// fields are set here.  Z: fused_parts + 1 arrays of n_steps*L*S*E floats; counters: route_fused_counter_words().
+// fields are set here.  Z: fused_parts arrays of n_steps*L*S*E floats; counters: route_fused_counter_words().
 cudaError_t route_fused_launch(RouterGemmPlan& plan, const mcce_config& c, const void* hidden, int n_steps, float* Z,
                                uint32_t* counters, RouteParams p, uint32_t* err, cudaStream_t st) {
   const uint64_t rows = (uint64_t)n_steps * c.n_layers * c.n_streams;
@@ -300,11 +263,10 @@ cudaError_t route_fused_launch(RouterGemmPlan& plan, const mcce_config& c, const
   args.tail_warps = (args.Sc * G + 31) / 32;
   const size_t n_tiles_all = (size_t)a.L * n_steps * a.n_tiles;
   args.Z = Z, args.z_stride = (size_t)rows * c.n_experts, args.err = err;
-  args.part_ready = counters, args.sum_ready = counters + 4 * n_tiles_all;
-  // the tail reads the summed logits only
-  p.n_steps = n_steps, p.hidden = nullptr, p.logits_in = Z + (size_t)a.KS * args.z_stride, p.n_partials = 1;
-  p.partial_stride = 0;
-  e = cudaMemsetAsync(counters, 0, 5 * n_tiles_all * sizeof(uint32_t), st);
+  args.part_ready = counters;
+  // the tail adds the K parts in the order 0 .. KS-1
+  p.n_steps = n_steps, p.hidden = nullptr, p.logits_in = Z, p.n_partials = a.KS, p.partial_stride = args.z_stride;
+  e = cudaMemsetAsync(counters, 0, n_tiles_all * sizeof(uint32_t), st);
   if (e != cudaSuccess) return e;
   Maps m;
   m.w = plan.w_res, m.x = plan.x_res, m.xt = plan.xt_res;
