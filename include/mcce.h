@@ -80,11 +80,16 @@ typedef struct {
   int32_t track_lifetime; /* 1: record how long experts stay cached (mcce_lifetime_stats)         */
   int32_t route_impl;     /* MCCE_ROUTE_AUTO (0) picks per launch what was measured faster;
                              MCCE_ROUTE_TWO_KERNELS: logits kernel, then routing tail;
-                             MCCE_ROUTE_FUSED: the single cooperative kernel wherever it can run       */
-  int32_t deterministic;  /* 1: y = sum_k w_k E_k(x) + shared experts is added in slot order on every path, so
-                             that repeated runs give identical bits (the paper's runs are deterministic,
-                             Sec. 4.1); the tensor-core path then writes one fp32 row per (stream, slot) and
-                             sums them in a second pass instead of adding into y with atomics              */
+                             MCCE_ROUTE_FUSED: the single cooperative kernel wherever it can run.  That kernel
+                             adds the parts of its split reduction of Eq. 3 in the order in which they arrive,
+                             so the last bit of a logit (and with it a selection between two experts whose
+                             logits are equal to within rounding) can differ between runs; the two-kernel path
+                             adds them in a fixed order.  The deterministic and the checked mode never use it */
+  int32_t deterministic;  /* 1: repeated runs give identical bits (the paper's runs are deterministic, Sec. 4.1):
+                             y = sum_k w_k E_k(x) + shared experts is added in slot order on every path (the
+                             tensor-core path then writes one fp32 row per (stream, slot) and sums them in a
+                             second pass instead of adding into y with atomics), and the router logits come
+                             from the two-kernel path                                                       */
   int32_t checked;        /* 1: checked mode.  Every routing launch is followed by kernels that verify the
                              logits (finite), the cache state (at most C resident experts per (stream,
                              layer), distinct recency keys) and every grouping pass (positions inside

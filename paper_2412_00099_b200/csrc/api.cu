@@ -12,11 +12,10 @@
 using namespace mcce;
 
 constexpr int kMaxPairs = 1024;
-// When MCCE_ROUTE_AUTO takes the single fused kernel: from four tokens per launch (for fewer the two launches are
-// faster) and while a CTA of it runs at most 12 tail warps.  With more, a thread has 80 registers, the tail
-// spills and becomes the slower chain.  Measured, eight tokens per launch, fused against two kernels:
-// Qwen-shaped (11 tail warps) 90 against 97 us, Mixtral-shaped (1) 60 against 85, OLMoE-shaped (16) 203 against 163.
-constexpr int kFusedMinTokens = 4, kFusedMaxTailWarps = 12;
+// When MCCE_ROUTE_AUTO takes the single fused kernel: from three tokens per launch.  Measured, fused against two
+// kernels, us per launch of 2 / 3 / 4 / 8 tokens: Qwen-shaped 39/37, 46/50, 55/62, 84/100; OLMoE-shaped 55/53,
+// 72/74, 84/97, 143/172; DeepSeek-shaped 47/44, 58/58, 69/73, 114/124; Mixtral-shaped 27/34, 33/43, 39/51, 60/85.
+constexpr int kFusedMinTokens = 3;
 
 struct mcce_ctx {
   mcce_config cfg;
@@ -62,6 +61,8 @@ struct mcce_ctx {
   RouterGemmPlan rg;
   void* wr_terms;
   float* z_buf;
+  float* z_acc;
+  size_t z_acc_bytes;
   uint32_t* z_ready;
   // optional per-kernel timing: event pairs recorded around each launch, summed by mcce_profile_read
   int profiling;
@@ -103,7 +104,7 @@ bool valid(const mcce_config* c) {
 
 struct Layout {
   size_t stamp, ever, sum_range, miss, cold, err, stats, offsets, perm, inv, offsets2, perm2, inv2, group_counts, Xg, Xg2, H, O, st_hidden, st_sel, st_w, st_y, st_hidden2, st_sel2, st_w2, st_y2,
-      wr_terms, z_buf, z_ready, load_tok, life, total;
+      wr_terms, z_buf, z_acc, z_ready, load_tok, life, total;
 };
 
 Layout layout_of(const mcce_config& c) {
@@ -151,6 +152,8 @@ Layout layout_of(const mcce_config& c) {
   // logits of up to router_gemm_steps_max() tokens; the router-resident kernels write one array per K part
   const size_t z_slots = (size_t)router_gemm_steps_max() * (router_gemm_res_applicable(c) ? router_gemm_res_parts_max() : 1);
   o.z_buf = take(rg ? z_slots * L * S * E * 4 : 0);
+  // the array the fused kernel accumulates a launch's logits in (zero between launches)
+  o.z_acc = take(rg ? (size_t)router_gemm_steps_max() * L * S * E * 4 : 0);
   o.z_ready = take(rg ? route_fused_counter_words((int)L, router_gemm_steps_max(), (int)S) * 4 : 0);   // counters of the fused kernel
   o.load_tok = take(c.track_lifetime ? L * S * E * 4 : 0);
   o.life = take(c.track_lifetime ? L * S * 3 * 8 : 0);
@@ -159,9 +162,12 @@ Layout layout_of(const mcce_config& c) {
 }
 
 bool use_fused(const mcce_ctx* ctx, int n_tokens) {
-  if (!ctx->rg.fused_ready || ctx->cfg.route_impl == MCCE_ROUTE_TWO_KERNELS) return false;
+  // (the checked mode looks at the logits after the routing pass: the fused kernel does not keep them; its
+  // logits are sums in order of arrival, which the deterministic mode rules out)
+  if (!ctx->rg.fused_ready || ctx->cfg.route_impl == MCCE_ROUTE_TWO_KERNELS || ctx->cfg.checked || ctx->cfg.deterministic)
+    return false;
   if (ctx->cfg.route_impl == MCCE_ROUTE_FUSED) return true;
-  return n_tokens >= kFusedMinTokens && ctx->rg.fused_tail_warps <= kFusedMaxTailWarps;
+  return n_tokens >= kFusedMinTokens;
 }
 
 int cuda_fail(mcce_ctx* ctx, cudaError_t e) {
@@ -267,13 +273,14 @@ extern "C" int mcce_create(const mcce_config* cfg, void* workspace, size_t works
   ctx->stage_w2 = (float*)(w + lo.st_w2), ctx->stage_y2 = (float*)(w + lo.st_y2);
   ctx->use_tc = cfg->ffn_impl != MCCE_FFN_SIMT && tc_applicable(*cfg);
   ctx->use_tc_router = router_gemm_applicable(*cfg);
-  ctx->wr_terms = w + lo.wr_terms, ctx->z_buf = (float*)(w + lo.z_buf), ctx->z_ready = (uint32_t*)(w + lo.z_ready);
+  ctx->wr_terms = w + lo.wr_terms, ctx->z_buf = (float*)(w + lo.z_buf), ctx->z_acc = (float*)(w + lo.z_acc), ctx->z_acc_bytes = lo.z_ready - lo.z_acc, ctx->z_ready = (uint32_t*)(w + lo.z_ready);
   ctx->load_tok = cfg->track_lifetime ? (uint32_t*)(w + lo.load_tok) : nullptr;
   ctx->life = cfg->track_lifetime ? (unsigned long long*)(w + lo.life) : nullptr;
   cudaError_t e = cudaSetDevice(cfg->device);
   // state arrays and the activation buffers start at zero (the slack rows must hold finite values)
   if (e == cudaSuccess) e = cudaMemset(w, 0, lo.O);
   if (e == cudaSuccess && cfg->track_lifetime) e = cudaMemset(w + lo.load_tok, 0, lo.total - lo.load_tok);
+  if (e == cudaSuccess && ctx->z_acc_bytes) e = cudaMemset(ctx->z_acc, 0, ctx->z_acc_bytes);
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
   if (e != cudaSuccess) {
     delete ctx;
@@ -369,6 +376,8 @@ extern "C" int mcce_reset(mcce_ctx* ctx, const int32_t* init_order, int keep_del
   CK(cudaMemset(ctx->miss, 0, LS * 4));
   CK(cudaMemset(ctx->cold, 0, LS * 4));
   CK(cudaMemset(ctx->err, 0, 64));
+  // a fused routing launch that gave up may have left sums behind
+  if (ctx->z_acc_bytes) CK(cudaMemset(ctx->z_acc, 0, ctx->z_acc_bytes));
   if (ctx->load_tok) {
     CK(cudaMemset(ctx->load_tok, 0, LS * E * 4));
     CK(cudaMemset(ctx->life, 0, LS * 3 * 8));
@@ -434,17 +443,11 @@ extern "C" int mcce_route_step(mcce_ctx* ctx, int32_t n_steps, const void* hidde
       if (use_fused(ctx, nt)) {
         cudaError_t fe = cudaSuccess;
         const int rc_f = timed(ctx, MCCE_K_ROUTE, st, [&]() {
-          fe = route_fused_launch(ctx->rg, c, h, nt, ctx->z_buf, ctx->z_ready, p, ctx->err, st);
+          fe = route_fused_launch(ctx->rg, c, h, nt, ctx->z_acc, ctx->z_ready, p, ctx->err, st);
           return fe == cudaErrorCooperativeLaunchTooLarge ? cudaSuccess : fe;
         });
         if (rc_f != MCCE_OK) return rc_f;
-        if (fe == cudaSuccess) {
-          if (c.checked) {
-            const int rc_c = check_after_route(ctx, ctx->z_buf, (size_t)ctx->rg.fused_parts * nt * LS * c.n_experts, st);
-            if (rc_c != MCCE_OK) return rc_c;
-          }
-          continue;
-        }
+        if (fe == cudaSuccess) continue;
         // the device cannot hold the whole grid at once (it is shared with other work): two kernels from now on
         cudaGetLastError();
         ctx->rg.fused_ready = 0;

@@ -4,18 +4,25 @@
 // next ones instead of following it in a second launch.
 //
 // A layer belongs to KS CTAs (one K part of the reduction each).  Warps 0-5 of a CTA are the GEMM (TMA
-// producer, MMA issuer, four epilogue warps); an epilogue warp stores the partial logits of its K part for its
-// 32 rows of the (token, stream tile) and then counts itself in on the tile's counter, after a device-wide
-// fence.  The remaining warps are the tail: the S streams of the layer are dealt out to its KS CTAs, a group of
-// lanes per stream as in route_group.cuh.  Before a token they wait (bounded) until all 4 x KS epilogue warps of
-// the layer have counted in on the tiles they read, then read the KS partial sums (L2-coherent loads) and add
-// them in the fixed order 0 .. KS-1.  The launch is cooperative, so every CTA that a tail warp waits for is
-// resident; the GEMM warps wait for nothing outside their CTA, so the waits cannot form a cycle.
+// producer, MMA issuer, four epilogue warps).  An epilogue warp adds the partial logits of its K part for its
+// 32 rows of the (token, stream tile) into the launch's logits array (fp32 reductions in L2; the array is zero
+// at launch) and notes its progress in shared memory.  Warp 6 publishes: once all four epilogue warps are
+// through with a pair it issues the device-wide fence and adds the CTA's four counts to the pair's counter.  (A
+// fence takes about 3 us while the device streams hidden states; issued by the epilogue warps themselves it
+// made them, not the tensor core, set the pace: 4.8 us per tile instead of 2.7.)  The remaining warps are the
+// tail: the S streams of the layer are dealt out to its KS CTAs, a group of lanes per stream as in
+// route_group.cuh.  Before a token they wait (bounded) until all KS CTAs of the layer have counted in on the
+// tiles they read, then read the sums (L2-coherent loads) and put the zeros back.  The launch is cooperative, so
+// every CTA that a tail warp waits for is resident; the GEMM warps and the publisher wait for nothing outside
+// their CTA, so the waits cannot form a cycle.
 //
-// Measured alternatives (Qwen-shaped, eight tokens per launch, this form: 90 us): holding the next token's KS
-// parts in registers while the current token is routed (64 more registers than the 96 a thread has here: spills,
-// 120 us); two more warps per CTA that add the parts up ahead of the tail, so that it reads one array (each
-// tile then passes through three more L2 round trips on two latency-bound warps: 164 us).
+// The order in which the KS parts of a logit are added is that of arrival: the last bit of a logit can differ
+// from run to run (the two-kernel path adds them in the fixed order 0 .. KS-1).
+//
+// Measured alternatives (Qwen-shaped, eight tokens per launch): one array per K part, read by the tail when the
+// token's turn comes (90 us); the same with the next token's parts held in registers while the current token is
+// routed (64 more registers than the 96 a thread has here: spills, 120 us); two more warps per CTA that add the
+// parts up ahead of the tail (three more L2 round trips per tile on two latency-bound warps: 164 us).
 #include "route_gemm_res.cuh"
 #include "route_group.cuh"
 
@@ -26,16 +33,21 @@ using namespace rres;
 namespace {
 
 constexpr int kGemmWarps = 6;      // TMA producer, MMA issuer, four epilogue warps
-constexpr int kFrontWarps = kGemmWarps;
+constexpr int kFrontWarps = kGemmWarps + 1;   // and the warp that publishes finished pairs
 constexpr int kMaxTailWarps = 16;
+// Hidden tiles in flight per CTA.  The stand-alone GEMM takes as many ring stages as fit; here a deeper ring
+// only lengthens the queues that the tail's loads, the counters and the publisher's fence wait behind (an L2
+// round trip takes 3-4 us while 5 stages per SM are in flight): Qwen-shaped, eight tokens, 5 stages 90 us,
+// 4 or 3 stages 84 us, 2 stages 95 us.
+constexpr int kFusedStages = 4;
 
 struct FusedArgs {
   Geometry g;
   int Sc;               // streams of the layer routed by each of its CTAs
   int tail_warps;
-  float* Z;             // [KS][n_steps, L, S, E] partial logits
-  size_t z_stride;
-  uint32_t* part_ready; // [L][n_steps * n_tiles] epilogue warps (4 per K part) that have stored their rows of a tile
+  float* Z;             // [n_steps, L, S, E] logits: zero at launch, the KS parts are added into it, the tail
+                        // reads them and puts the zeros back
+  uint32_t* part_ready; // [L][n_steps * n_tiles] epilogue warps (4 per K part) whose rows of a tile are added in
   uint32_t* err;
 };
 
@@ -83,11 +95,13 @@ struct TailSync {
       if (!wait_count(ready_l + t * n_tiles + tile, target, abort_flag, err, 36u)) return false;
     return true;
   }
-  __device__ __forceinline__ bool ready(int t) const {
-    bool ok = true;
-    for (int tile = tile_lo; tile <= tile_hi; ++tile) ok = ok && ld_acquire(ready_l + t * n_tiles + tile) >= target;
-    return __all_sync(kFull, ok);
+  // a warp's streams are adjacent: they lie in one tile or in two
+  uint32_t c_lo, c_hi;
+  __device__ __forceinline__ void probe(int t) {
+    c_lo = ld_acquire(ready_l + t * n_tiles + tile_lo);
+    c_hi = ld_acquire(ready_l + t * n_tiles + tile_hi);
   }
+  __device__ __forceinline__ bool probed_ok() const { return __all_sync(kFull, c_lo >= target && c_hi >= target); }
 };
 
 // TW: tail warps the kernel is compiled for (its register budget follows from the thread count).
@@ -115,16 +129,45 @@ route_fused_kernel(const __grid_constant__ Maps maps, const FusedArgs args, cons
     if (lane == 0) issue_mmas(a, m, tmem_base, kp, 0, 1, args.err, 31u);
   } else if (warp < kGemmWarps) {
     const int quad = warp & 3, row = quad * 32 + lane;
-    float* Zp = args.Z + (size_t)ks * args.z_stride;
     for (int i = 0; i < n_pairs; ++i) {
       const int t = i / a.n_tiles, tile = i % a.n_tiles;
       const size_t grow = (size_t)(t * a.L + l) * a.S + tile * kTileM + row;
       const bool row_ok = tile * kTileM + row < a.S;
-      if (!drain_pair(a, m, tmem_base, kp, (uint32_t)i, quad, lane, Zp + grow * a.E, row_ok, args.err, 35u)) break;
-      uint32_t* cnt = args.part_ready + (size_t)l * n_pairs + i;
-      __threadfence();   // this lane's part of the tile is visible device-wide before the warp counts in
+      if (!drain_pair<true>(a, m, tmem_base, kp, (uint32_t)i, quad, lane, args.Z + grow * a.E, row_ok, args.err, 35u)) break;
+      // this warp's additions of pair i are ordered before its progress word for the other warps of the CTA
+      asm volatile("fence.acq_rel.cta;" ::: "memory");
       __syncwarp();
-      if (lane == 0) atomicAdd(cnt, 1u);
+      if (lane == 0) {
+        asm volatile("fence.acq_rel.cta;" ::: "memory");
+        m.drained[quad] = (uint32_t)i + 1u;
+      }
+    }
+  } else if (warp == kGemmWarps) {
+    // ---- publisher: pairs that all four epilogue warps have finished are counted in device-wide -------------
+    if (lane == 0) {
+      uint32_t* cnt = args.part_ready + (size_t)l * n_pairs;
+      uint32_t published = 0u;
+      unsigned long long last = global_ns();
+      for (uint32_t it = 1; published < (uint32_t)n_pairs; ++it) {
+        const uint32_t d = min(min(m.drained[0], m.drained[1]), min(m.drained[2], m.drained[3]));
+        if (d > published) {
+          // acquire on the progress words, release for the counters: the epilogue warps' additions come first
+          asm volatile("fence.acq_rel.gpu;" ::: "memory");
+          for (uint32_t i = published; i < d; ++i) atomicAdd(cnt + i, 4u);
+          published = d;
+          last = global_ns();
+          continue;
+        }
+        __nanosleep(100);
+        if ((it & 63u) == 0u) {
+          if (*m.abort_flag) break;
+          if (global_ns() - last > kWaitLimitNs) {
+            *m.abort_flag = 1u;
+            atomicCAS(args.err, 0u, 37u);
+            break;
+          }
+        }
+      }
     }
   } else {
     // ---- routing tail of this CTA's share of the layer's streams -------------------------------------------
@@ -136,8 +179,8 @@ route_fused_kernel(const __grid_constant__ Maps maps, const FusedArgs args, cons
       sync.ready_l = args.part_ready + (size_t)l * n_pairs, sync.n_tiles = a.n_tiles, sync.target = 4u * (uint32_t)a.KS;
       sync.tile_lo = min(a.S - 1, ks * args.Sc + (tw * 32) / G) / kTileM;
       sync.tile_hi = min(a.S - 1, ks * args.Sc + min(args.Sc - 1, (tw * 32 + 31) / G)) / kTileM;
-      sync.abort_flag = m.abort_flag, sync.err = args.err;
-      rgroup::route_group_streams<G, KMAX, rgroup::kLoadDirect, 1, true>(p, l, s_raw, lane % G, sync);
+      sync.abort_flag = m.abort_flag, sync.err = args.err, sync.c_lo = sync.c_hi = 0u;
+      rgroup::route_group_streams<G, KMAX, rgroup::kPrefetchReady, 1, true, true>(p, l, s_raw, lane % G, sync);
     }
   }
   teardown(m, tmem_base, warp, 1);
@@ -257,15 +300,14 @@ cudaError_t route_fused_launch(RouterGemmPlan& plan, const mcce_config& c, const
   a.KS = plan.fused_parts, a.slabs = c.d_model / kTileK;
   a.n_tiles = (c.n_streams + kTileM - 1) / kTileM;
   a.res_bytes = res_bytes_of(a.slabs, a.KS, a.Epad);
-  a.n_stages = stages_of(a.res_bytes);
+  a.n_stages = stages_of(a.res_bytes) < kFusedStages ? stages_of(a.res_bytes) : kFusedStages;
   const int G = group_of(c.n_experts);
   args.Sc = (c.n_streams + a.KS - 1) / a.KS;
   args.tail_warps = (args.Sc * G + 31) / 32;
   const size_t n_tiles_all = (size_t)a.L * n_steps * a.n_tiles;
-  args.Z = Z, args.z_stride = (size_t)rows * c.n_experts, args.err = err;
+  args.Z = Z, args.err = err;
   args.part_ready = counters;
-  // the tail adds the K parts in the order 0 .. KS-1
-  p.n_steps = n_steps, p.hidden = nullptr, p.logits_in = Z, p.n_partials = a.KS, p.partial_stride = args.z_stride;
+  p.n_steps = n_steps, p.hidden = nullptr, p.logits_in = Z, p.n_partials = 1, p.partial_stride = 0;
   e = cudaMemsetAsync(counters, 0, n_tiles_all * sizeof(uint32_t), st);
   if (e != cudaSuccess) return e;
   Maps m;

@@ -85,7 +85,7 @@ __device__ __forceinline__ float group_sum(float v) {
 
 
 // Loads of logits: through the read-only path when another kernel wrote them, L2-coherent when CTAs of the
-// running kernel did.
+// running kernel did (ACCUM below).
 template <bool COHERENT>
 __device__ __forceinline__ float4 ldz4(const float4* q) { return COHERENT ? __ldcg(q) : __ldg(q); }
 template <bool COHERENT>
@@ -104,26 +104,33 @@ constexpr int kLoadDirect = 0;     // loaded when the token's turn comes (after 
 constexpr int kPrefetchAll = 1;    // every token is there already: the next token's logits are requested while
                                    // the current one is routed
 constexpr int kPrefetchReady = 2;  // tokens appear while the kernel runs: the next token's logits are requested
-                                   // early if sync.ready(t + 1) says they are there, else after sync.wait(t + 1)
+                                   // half-way through the current one if they are there by then (sync.probe(t + 1)
+                                   // before the selection, sync.probed_ok() after it), else after sync.wait(t + 1)
 
 // For callers whose logits are all there before the launch.
 struct AllPresent {
   __device__ __forceinline__ bool wait(int) const { return true; }
-  __device__ __forceinline__ bool ready(int) const { return true; }
+  __device__ __forceinline__ void probe(int) {}
+  __device__ __forceinline__ bool probed_ok() const { return true; }
 };
 
 // Routes the p.n_steps tokens of stream s_raw of layer l.  All 32 lanes of a warp must call this together
 // (groups past the last stream run on stream 0's data and store nothing).  `sub` is the lane's index in its
 // group.  sync.wait(t) is called by every lane before the logits of token t are read and returns false to give
-// up; sync.ready(t) asks without waiting whether they can be read (both: the same answer in all lanes of a warp).
+// up; sync.probe(t) starts asking, without waiting, whether they can be read, and sync.probed_ok() has the answer
+// (the same one in all lanes of a warp).
+//
+// ACCUM: the logits are sums that CTAs of the running kernel accumulate in an array that is zero between launches
+// (one array: p.n_partials == 1).  They are read L2-coherently, and the lanes that own a row put the zeros back.
 //
 // A token's work has a part that does not depend on the cache (logits, range statistic, bias, top-J: stage A)
 // and a part that does (promotion, top-K, misses, LRU: stage B); only B is a chain from token to token.
 // With a prefetching MODE up to NP partial logit arrays of the next token are held in registers.
-template <int G, int KMAX, int MODE, int NP, bool COHERENT, typename Sync>
+template <int G, int KMAX, int MODE, int NP, bool COHERENT, bool ACCUM, typename Sync>
 __device__ __forceinline__ void route_group_streams(const RouteParams& p, const int l, const int s_raw, const int sub,
                                                     Sync sync) {
   constexpr bool PF = MODE != kLoadDirect;
+  static_assert(!ACCUM || (COHERENT && PF && NP == 1), "accumulated logits are one array, cleared where it is prefetched");
   const bool active = s_raw < p.S;
   const int s = active ? s_raw : 0;
   const size_t pair = (size_t)l * p.S + s;
@@ -151,60 +158,59 @@ __device__ __forceinline__ void route_group_streams(const RouteParams& p, const 
   }
   sum_range = p.sum_range[pair];
 
+  // Where this lane's eight logits of token t start in a logits array.
+  auto z_at = [&](int t) -> const float* { return p.logits_in + (((size_t)t * p.L + l) * p.S + s) * E + e0; };
+  auto load8 = [&](const float* src, float (&v)[kNE]) {
+    if (vec4) {
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        float4 u = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (e0 + 4 * h < E) u = ldz4<COHERENT>((const float4*)(src + 4 * h));
+        v[4 * h] = u.x, v[4 * h + 1] = u.y, v[4 * h + 2] = u.z, v[4 * h + 3] = u.w;
+      }
+    } else {
+#pragma unroll
+      for (int i = 0; i < kNE; ++i) v[i] = e0 + i < E ? ldz1<COHERENT>(src + i) : 0.f;
+    }
+  };
+
   // The partial logits of the next token are requested before the current token is routed, so that their
   // latency (L2, mostly) is off the critical path: up to NP parts of eight logits per lane in flight.
-  float4 raw[PF ? NP : 1][2];
+  float raw[PF ? NP : 1][kNE];
   auto request = [&](int t) {
-    const float* src = p.logits_in + (((size_t)t * p.L + l) * p.S + s) * E + e0;
+    const float* src = z_at(t);
 #pragma unroll
     for (int q = 0; q < (PF ? NP : 1); ++q)
+      if (q < p.n_partials) load8(src + (size_t)q * p.partial_stride, raw[q]);
+    if (ACCUM && active) {
+      // same thread, same addresses: the loads above are ordered before these stores
 #pragma unroll
       for (int h = 0; h < 2; ++h)
-        if (q < p.n_partials && e0 + 4 * h < E) raw[q][h] = ldz4<COHERENT>((const float4*)(src + (size_t)q * p.partial_stride + 4 * h));
+        if (e0 + 4 * h < E) __stcg((float4*)const_cast<float*>(src + 4 * h), make_float4(0.f, 0.f, 0.f, 0.f));
+    }
   };
 
   // ---- stage A: logits of token t (the K parts of the router GEMM summed in a fixed order), Eq. 8, top-J -------
   auto stage_a = [&](const int t, Pre& o) {
     const size_t row = ((size_t)t * p.L + l) * p.S + s;
     float (&z)[kNE] = o.z;
-    const float* src = p.logits_in + row * E + e0;
     if (PF) {
 #pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (e0 + 4 * h < E) {
-          v = raw[0][h];
+      for (int i = 0; i < kNE; ++i) {
+        float v = raw[0][i];
 #pragma unroll
-          for (int q = 1; q < (PF ? NP : 1); ++q)
-            if (q < p.n_partials) {
-              const float4 u = raw[q][h];
-              v.x = __fadd_rn(v.x, u.x), v.y = __fadd_rn(v.y, u.y), v.z = __fadd_rn(v.z, u.z), v.w = __fadd_rn(v.w, u.w);
-            }
-        }
-        z[4 * h] = v.x, z[4 * h + 1] = v.y, z[4 * h + 2] = v.z, z[4 * h + 3] = v.w;
-      }
-    } else if (vec4) {
-#pragma unroll
-      for (int i = 0; i < kNE; i += 4) {
-        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (e0 + i < E) {
-          v = ldz4<COHERENT>((const float4*)(src + i));
-          for (int q = 1; q < p.n_partials; ++q) {
-            const float4 u = ldz4<COHERENT>((const float4*)(src + (size_t)q * p.partial_stride + i));
-            v.x = __fadd_rn(v.x, u.x), v.y = __fadd_rn(v.y, u.y), v.z = __fadd_rn(v.z, u.z), v.w = __fadd_rn(v.w, u.w);
-          }
-        }
-        z[i] = v.x, z[i + 1] = v.y, z[i + 2] = v.z, z[i + 3] = v.w;
+        for (int q = 1; q < (PF ? NP : 1); ++q)
+          if (q < p.n_partials) v = __fadd_rn(v, raw[q][i]);
+        z[i] = v;
       }
     } else {
+      const float* src = z_at(t);
+      load8(src, z);
+      for (int q = 1; q < p.n_partials; ++q) {
+        float u[kNE];
+        load8(src + (size_t)q * p.partial_stride, u);
 #pragma unroll
-      for (int i = 0; i < kNE; ++i) {
-        float v = 0.f;
-        if (e0 + i < E) {
-          v = ldz1<COHERENT>(src + i);
-          for (int q = 1; q < p.n_partials; ++q) v = __fadd_rn(v, ldz1<COHERENT>(src + (size_t)q * p.partial_stride + i));
-        }
-        z[i] = v;
+        for (int i = 0; i < kNE; ++i) z[i] = __fadd_rn(z[i], u[i]);
       }
     }
     if (p.logits_out != nullptr && active) {
@@ -249,7 +255,7 @@ __device__ __forceinline__ void route_group_streams(const RouteParams& p, const 
   };
 
   // ---- stage B: Eq. 7, top-K, weights, Eq. 4, LRU ---------------------------------------------------------------------
-  auto stage_b = [&](const int t, const Pre& in) {
+  auto stage_b = [&](const int t, const Pre& in, auto&& after_selection) {
     const size_t row = ((size_t)t * p.L + l) * p.S + s;
     const float (&z)[kNE] = in.z;
     const float zmax = in.zmax, bias = in.bias;
@@ -292,6 +298,7 @@ __device__ __forceinline__ void route_group_streams(const RouteParams& p, const 
         }
       }
     }
+    after_selection();
     {
       const uint32_t both = group_or<G>(miss_bits | (cold_bits << 16));
       miss_bits = both & 0xffffu, cold_bits = both >> 16;
@@ -379,11 +386,15 @@ __device__ __forceinline__ void route_group_streams(const RouteParams& p, const 
     Pre pre;
     stage_a(t, pre);            // with PF: consumes the registers that request(t) filled
     bool requested = false;
-    if (PF && t + 1 < p.n_steps) {
-      requested = MODE == kPrefetchAll || sync.ready(t + 1);
-      if (requested) request(t + 1);
-    }
-    stage_b(t, pre);
+    const bool more = PF && t + 1 < p.n_steps;
+    if (more && MODE == kPrefetchAll) request(t + 1), requested = true;
+    if (more && MODE == kPrefetchReady) sync.probe(t + 1);
+    stage_b(t, pre, [&]() {
+      if (more && MODE == kPrefetchReady) {
+        requested = sync.probed_ok();
+        if (requested) request(t + 1);
+      }
+    });
     if (PF && t + 1 < p.n_steps && !requested) {
       alive = sync.wait(t + 1);
       if (alive) request(t + 1);

@@ -17,7 +17,7 @@ __global__ void __launch_bounds__(kThreads) route_group_kernel(const RouteParams
   const int blocks_per_layer = (p.S + kPerCta - 1) / kPerCta;
   const int l = blockIdx.x / blocks_per_layer;
   const int s_raw = (blockIdx.x % blocks_per_layer) * kPerCta + threadIdx.x / G;
-  rgroup::route_group_streams<G, KMAX, PF ? rgroup::kPrefetchAll : rgroup::kLoadDirect, kPartsMax, false>(
+  rgroup::route_group_streams<G, KMAX, PF ? rgroup::kPrefetchAll : rgroup::kLoadDirect, kPartsMax, false, false>(
       p, l, s_raw, threadIdx.x % G, rgroup::AllPresent());
 }
 

@@ -160,16 +160,24 @@ def test_fused_kernel_and_two_kernel_path_leave_the_same_state():
 
 
 def test_automatic_choice_of_the_routing_kernels():
-    """MCCE_ROUTE_AUTO: the fused kernel from four tokens per launch while a CTA of it needs at most 12 tail warps
-    (few streams per CTA or few experts), the two kernels otherwise."""
+    """MCCE_ROUTE_AUTO: the fused kernel from three tokens per launch where the configuration has one, the two
+    kernels otherwise."""
     for base, kw, n, want in ((synth.MIXTRAL, dict(L=32, S=64, d=1024), 8, mb.ROUTER_FUSED),
                               (synth.MIXTRAL, dict(L=32, S=64, d=1024), 1, mb.ROUTER_RESIDENT_TAIL),
                               (synth.QWEN, dict(L=24, S=64, d=512), 8, mb.ROUTER_FUSED),
-                              (synth.OLMOE, dict(L=16, S=512, d=512), 8, mb.ROUTER_RESIDENT_TAIL),
+                              (synth.OLMOE, dict(L=16, S=512, d=512), 8, mb.ROUTER_FUSED),
+                              (synth.OLMOE, dict(L=16, S=512, d=512), 2, mb.ROUTER_RESIDENT_TAIL),
                               (synth.QWEN, dict(L=2, S=16, d=256, E=100), 8, mb.ROUTER_GEMM_TAIL),
                               (synth.TINY, dict(), 8, mb.ROUTER_FP32_PIPE)):
         wl = base.with_(**kw)
         eng = mb.engine_for(wl, ffn_impl=mb.FFN_SIMT)
         eng.set_router(H.to_dev(wl.router()))
         assert eng.router_kernel_kind(n) == want, (wl.name, n)
+        eng.close()
+    # the fused kernel adds the parts of a logit in order of arrival: not in the deterministic or the checked mode
+    wl = synth.QWEN.with_(L=24, S=64, d=512)
+    for kw in (dict(deterministic=1), dict(checked=1)):
+        eng = mb.engine_for(wl, ffn_impl=mb.FFN_SIMT, route_impl=mb.ROUTE_FUSED, **kw)
+        eng.set_router(H.to_dev(wl.router()))
+        assert eng.router_kernel_kind(8) == mb.ROUTER_RESIDENT_TAIL, kw
         eng.close()
