@@ -62,7 +62,7 @@ struct mcce_ctx {
   void* wr_terms;
   float* z_buf;
   float* z_acc;
-  size_t z_acc_bytes;
+  size_t z_acc_bytes;   // the accumulation array and, behind it, the counters of the fused routing kernel
   uint32_t* z_ready;
   // optional per-kernel timing: event pairs recorded around each launch, summed by mcce_profile_read
   int profiling;
@@ -273,7 +273,7 @@ extern "C" int mcce_create(const mcce_config* cfg, void* workspace, size_t works
   ctx->stage_w2 = (float*)(w + lo.st_w2), ctx->stage_y2 = (float*)(w + lo.st_y2);
   ctx->use_tc = cfg->ffn_impl != MCCE_FFN_SIMT && tc_applicable(*cfg);
   ctx->use_tc_router = router_gemm_applicable(*cfg);
-  ctx->wr_terms = w + lo.wr_terms, ctx->z_buf = (float*)(w + lo.z_buf), ctx->z_acc = (float*)(w + lo.z_acc), ctx->z_acc_bytes = lo.z_ready - lo.z_acc, ctx->z_ready = (uint32_t*)(w + lo.z_ready);
+  ctx->wr_terms = w + lo.wr_terms, ctx->z_buf = (float*)(w + lo.z_buf), ctx->z_acc = (float*)(w + lo.z_acc), ctx->z_acc_bytes = lo.load_tok - lo.z_acc, ctx->z_ready = (uint32_t*)(w + lo.z_ready);
   ctx->load_tok = cfg->track_lifetime ? (uint32_t*)(w + lo.load_tok) : nullptr;
   ctx->life = cfg->track_lifetime ? (unsigned long long*)(w + lo.life) : nullptr;
   cudaError_t e = cudaSetDevice(cfg->device);
@@ -376,7 +376,7 @@ extern "C" int mcce_reset(mcce_ctx* ctx, const int32_t* init_order, int keep_del
   CK(cudaMemset(ctx->miss, 0, LS * 4));
   CK(cudaMemset(ctx->cold, 0, LS * 4));
   CK(cudaMemset(ctx->err, 0, 64));
-  // a fused routing launch that gave up may have left sums behind
+  // a fused routing launch that gave up may have left sums and counts behind (the counters follow the sums)
   if (ctx->z_acc_bytes) CK(cudaMemset(ctx->z_acc, 0, ctx->z_acc_bytes));
   if (ctx->load_tok) {
     CK(cudaMemset(ctx->load_tok, 0, LS * E * 4));

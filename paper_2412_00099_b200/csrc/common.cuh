@@ -93,6 +93,7 @@ struct RouterGemmPlan {
   int res_parts_single;       // the same for a launch of one layer at a time
   int fused_ready, fused_parts;   // the same for the kernel that also runs the routing tail (route_fused.cu)
   int fused_tail_warps;           // tail warps per CTA of that kernel
+  int fused_flip;                 // which of its two counter sets the next launch uses
 };
 bool router_gemm_applicable(const mcce_config& c);
 int router_gemm_steps_max();

@@ -48,6 +48,8 @@ struct FusedArgs {
   float* Z;             // [n_steps, L, S, E] logits: zero at launch, the KS parts are added into it, the tail
                         // reads them and puts the zeros back
   uint32_t* part_ready; // [L][n_steps * n_tiles] epilogue warps (4 per K part) whose rows of a tile are added in
+  uint32_t* next_ready; // the counters of the next launch (the two sets alternate): cleared by this one
+  int counter_words;    // words of a set
   uint32_t* err;
 };
 
@@ -118,6 +120,8 @@ route_fused_kernel(const __grid_constant__ Maps maps, const FusedArgs args, cons
 
   if (threadIdx.x == 0) init_barriers(m);
   if (warp == 1) tmem_alloc(smem_u32(m.tmem_slot), kTmemCols);
+  for (int w = blockIdx.x * blockDim.x + threadIdx.x; w < args.counter_words; w += gridDim.x * blockDim.x)
+    args.next_ready[w] = 0u;
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -247,9 +251,10 @@ cudaError_t launch_any(int G, int K, int TW, const Maps& m, const FusedArgs& a, 
 
 }  // namespace
 
-// Counters the kernel needs per launch: one word per (layer, token, stream tile).
+// Counter words the kernel needs: one per (layer, token, stream tile), in two sets that alternate from launch to
+// launch (a launch clears the set of the next one; both start at zero).
 size_t route_fused_counter_words(int n_layers, int n_steps, int n_streams) {
-  return (size_t)n_layers * n_steps * ((n_streams + kTileM - 1) / kTileM);
+  return 2 * (size_t)n_layers * n_steps * ((n_streams + kTileM - 1) / kTileM);
 }
 
 // Fixes the K-split of the fused kernel for this configuration, or leaves plan->fused_ready at 0 when the two-kernel
@@ -287,7 +292,8 @@ int route_fused_plan(const mcce_config& c, RouterGemmPlan* plan) {
 }
 
 // The routing step of n_steps tokens of all layers.  p carries the routing parameters and outputs; its logits
-// fields are set here.  Z: fused_parts arrays of n_steps*L*S*E floats; counters: route_fused_counter_words().
+// fields are set here.  Z: n_steps*L*S*E floats, zero; counters: route_fused_counter_words() words for the largest
+// n_steps, zero before the first launch.
 cudaError_t route_fused_launch(RouterGemmPlan& plan, const mcce_config& c, const void* hidden, int n_steps, float* Z,
                                uint32_t* counters, RouteParams p, uint32_t* err, cudaStream_t st) {
   const uint64_t rows = (uint64_t)n_steps * c.n_layers * c.n_streams;
@@ -304,15 +310,18 @@ cudaError_t route_fused_launch(RouterGemmPlan& plan, const mcce_config& c, const
   const int G = group_of(c.n_experts);
   args.Sc = (c.n_streams + a.KS - 1) / a.KS;
   args.tail_warps = (args.Sc * G + 31) / 32;
-  const size_t n_tiles_all = (size_t)a.L * n_steps * a.n_tiles;
   args.Z = Z, args.err = err;
-  args.part_ready = counters;
+  // the two counter sets alternate; a set holds the words of the largest launch
+  const size_t set_words = route_fused_counter_words(c.n_layers, router_gemm_steps_max(), c.n_streams) / 2;
+  args.part_ready = counters + (size_t)(plan.fused_flip & 1) * set_words;
+  args.next_ready = counters + (size_t)((plan.fused_flip & 1) ^ 1) * set_words;
+  args.counter_words = (int)set_words;
   p.n_steps = n_steps, p.hidden = nullptr, p.logits_in = Z, p.n_partials = 1, p.partial_stride = 0;
-  e = cudaMemsetAsync(counters, 0, n_tiles_all * sizeof(uint32_t), st);
-  if (e != cudaSuccess) return e;
   Maps m;
   m.w = plan.w_res, m.x = plan.x_res, m.xt = plan.xt_res;
-  return launch_any(G, c.top_k, tail_bucket(args.tail_warps), m, args, p, st);
+  e = launch_any(G, c.top_k, tail_bucket(args.tail_warps), m, args, p, st);
+  if (e == cudaSuccess) plan.fused_flip ^= 1;
+  return e;
 }
 
 }  // namespace mcce
