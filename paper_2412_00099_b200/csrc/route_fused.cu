@@ -138,12 +138,16 @@ route_fused_kernel(const __grid_constant__ Maps maps, const FusedArgs args, cons
       const size_t grow = (size_t)(t * a.L + l) * a.S + tile * kTileM + row;
       const bool row_ok = tile * kTileM + row < a.S;
       if (!drain_pair<true>(a, m, tmem_base, kp, (uint32_t)i, quad, lane, args.Z + grow * a.E, row_ok, args.err, 35u)) break;
-      // this warp's additions of pair i are ordered before its progress word for the other warps of the CTA
-      asm volatile("fence.acq_rel.cta;" ::: "memory");
-      __syncwarp();
-      if (lane == 0) {
+      // Once per token (after its last stream tile; the tail consumes whole tokens): this warp's additions of the
+      // token's pairs are ordered before its progress word for the other warps of the CTA.  The fence waits until
+      // the reductions have been performed in L2, a round trip of 2-3 us here.
+      if (tile == a.n_tiles - 1) {
         asm volatile("fence.acq_rel.cta;" ::: "memory");
-        m.drained[quad] = (uint32_t)i + 1u;
+        __syncwarp();
+        if (lane == 0) {
+          asm volatile("fence.acq_rel.cta;" ::: "memory");
+          m.drained[quad] = (uint32_t)i + 1u;
+        }
       }
     }
   } else if (warp == kGemmWarps) {
@@ -297,7 +301,7 @@ int route_fused_plan(const mcce_config& c, RouterGemmPlan* plan) {
 cudaError_t route_fused_launch(RouterGemmPlan& plan, const mcce_config& c, const void* hidden, int n_steps, float* Z,
                                uint32_t* counters, RouteParams p, uint32_t* err, cudaStream_t st) {
   const uint64_t rows = (uint64_t)n_steps * c.n_layers * c.n_streams;
-  cudaError_t e = hidden_maps(plan, hidden, rows, c.d_model);
+  cudaError_t e = hidden_maps(plan, hidden, rows, c.d_model, c.n_streams);
   if (e != cudaSuccess) return e;
   FusedArgs args;
   Geometry& a = args.g;

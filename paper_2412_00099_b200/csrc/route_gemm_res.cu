@@ -112,7 +112,7 @@ cudaError_t router_gemm_res_launch(RouterGemmPlan& plan, const mcce_config& c, c
   cudaError_t e0 = sm_count_and_smem_optin(router_gemm_res_kernel, (size_t)kSmemMax + 1024, cache, &sms);
   if (e0 != cudaSuccess) return e0;
   const uint64_t rows = (uint64_t)n_steps * Ls * c.n_streams;
-  e0 = hidden_maps(plan, hidden, rows, c.d_model);
+  e0 = hidden_maps(plan, hidden, rows, c.d_model, c.n_streams);
   if (e0 != cudaSuccess) return e0;
   ResArgs args;
   Geometry& a = args.g;

@@ -41,7 +41,8 @@ struct Geometry {
 };
 struct Maps {
   CUtensorMap w;   // 3-D: [3*L][E][d] bf16 terms (term-major), box 1 x Epad x 64
-  CUtensorMap x;   // 2-D: [n_steps*L*S][d] hidden rows, box 16 x 64 (ragged last tile of a layer)
+  CUtensorMap x;   // 2-D: [n_steps*L*S][d] hidden rows, box (S mod 128, rounded up to 16) x 64: the ragged last
+                   // tile of a layer in one copy (several small copies per slab cost more than the bytes they save)
   CUtensorMap xt;  // the same rows, box 128 x 64 (full tiles)
 };
 
@@ -133,17 +134,13 @@ __device__ __forceinline__ void produce(const Maps& maps, const Geometry& a, con
   for (int i = first; i < n_pairs; i += step) {
     const int t = i / a.n_tiles, tile = i % a.n_tiles;
     const int row0 = (t * a.L + l) * a.S + tile * kTileM;
+    // rows of the copy: a whole tile, or the ragged last tile of the layer rounded up to the box of maps.x
     const int n_box = (min(kTileM, a.S - tile * kTileM) + kXBox - 1) / kXBox;
     for (int j = 0; j < kp.n_k; ++j) {
       if (!mbar_wait(m.bar_empty + 8 * stage, phase ^ 1u, m.abort_flag, err, code0)) return;
       const uint32_t sa = m.ring + stage * kStageBytes, full = m.bar_full + 8 * stage;
       mbar_expect_tx(full, (uint32_t)n_box * kXBox * kRowBytes);
-      if (n_box == kTileM / kXBox) {   // one 16 KB copy: measurably faster than eight of 2 KB
-        tma_load_2d(sa, &maps.xt, (kp.k_begin + j) * kTileK, row0, full);
-      } else {
-        for (int b = 0; b < n_box; ++b)
-          tma_load_2d(sa + b * kXBox * kRowBytes, &maps.x, (kp.k_begin + j) * kTileK, row0 + b * kXBox, full);
-      }
+      tma_load_2d(sa, n_box == kTileM / kXBox ? &maps.xt : &maps.x, (kp.k_begin + j) * kTileK, row0, full);
       if (++stage == (uint32_t)a.n_stages) stage = 0, phase ^= 1u;
     }
   }
@@ -253,12 +250,13 @@ __device__ __forceinline__ void teardown(const Smem& m, uint32_t tmem_base, int 
 }
 
 // Host side: tensor maps over the hidden rows of a launch (rebuilt when the pointer or the row count changes).
-inline cudaError_t hidden_maps(RouterGemmPlan& plan, const void* hidden, uint64_t rows, int d_model) {
+inline cudaError_t hidden_maps(RouterGemmPlan& plan, const void* hidden, uint64_t rows, int d_model, int n_streams) {
   if (plan.hidden_ptr_res == hidden && plan.hidden_rows_res == rows) return cudaSuccess;
   EncodeFn fn = encode_fn();
   const cuuint64_t dims[2] = {(cuuint64_t)d_model, rows};
   const cuuint64_t strides[1] = {(cuuint64_t)d_model * 2};
-  const cuuint32_t box[2] = {(cuuint32_t)kTileK, (cuuint32_t)kXBox};
+  const int ragged = n_streams % kTileM ? ((n_streams % kTileM + kXBox - 1) / kXBox) * kXBox : kXBox;
+  const cuuint32_t box[2] = {(cuuint32_t)kTileK, (cuuint32_t)ragged};
   const cuuint32_t box_tile[2] = {(cuuint32_t)kTileK, (cuuint32_t)kTileM};
   const cuuint32_t estr[2] = {1, 1};
   if (!fn || fn(&plan.x_res, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(hidden), dims, strides, box, estr,
