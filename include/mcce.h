@@ -34,7 +34,9 @@ enum {
   MCCE_ENOSPC = -2,   /* workspace too small                                            */
   MCCE_ESTATE = -3,   /* weights not set, or a counter would overflow (reset needed)    */
   MCCE_ECUDA = -4,    /* a CUDA call failed; see mcce_last_cuda_error                   */
-  MCCE_ETIMEOUT = -5, /* a bounded wait inside a kernel gave up; the context stays usable */
+  MCCE_ETIMEOUT = -5, /* a bounded wait inside a kernel gave up: the launch it happened in is incomplete (results,
+                         cache state and internal buffers), the CUDA context stays usable; mcce_reset brings the
+                         mcce context back to a defined state                                             */
   MCCE_ELIMIT = -6,   /* problem larger than the fixed array of mcce_route_trace_static   */
   MCCE_EINDEX = -7,   /* an expert id outside [0, E) reached the grouping pass (the pair was skipped), or a
                          check of the checked mode failed: a grouping position outside [0, S*K), more than C

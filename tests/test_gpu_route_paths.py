@@ -60,13 +60,15 @@ def test_group_tail_and_warp_tail_agree_bit_for_bit():
 
 
 def follow_chunked(eng, o, Wr, xs, chunk, kind):
-    """check_route_follow with `chunk` tokens per launch."""
+    """check_route_follow with `chunk` tokens per launch (a list: the lengths of successive launches)."""
     T = xs.shape[0]
     xd = torch.from_numpy(xs.view(np.int16)).cuda().view(torch.bfloat16)
-    near, max_dz, t = 0, 0.0, 0
+    near, max_dz, t, i = 0, 0.0, 0, 0
     while t < T:
-        n = min(chunk, T - t)
-        assert eng.router_kernel_kind(n) == kind
+        n = min(chunk[i % len(chunk)] if isinstance(chunk, (list, tuple)) else chunk, T - t)
+        i += 1
+        if kind is not None:
+            assert eng.router_kernel_kind(n) == kind
         sel, w, zg = (a.cpu().numpy() for a in eng.route_step(hidden=xd[t:t + n], n_steps=n, want_logits=True))
         for i in range(n):
             z_own = o.logits(Wr, xs[t + i])
@@ -128,6 +130,24 @@ def test_router_resident_gemm_then_tail(base, kw):
     near, dz = follow_chunked(eng, o, Wr, xs[:8], 8, mb.ROUTER_RESIDENT_TAIL)
     near2, dz2 = follow_chunked(eng, o, Wr, xs[8:], 1, mb.ROUTER_RESIDENT_TAIL)
     print("%s resident: %d near ties, max logit err %.2e" % (wl.name, near + near2, max(dz, dz2)))
+    eng.close()
+
+
+def test_fused_launches_of_varying_length_and_a_reset_in_between():
+    """The fused kernel accumulates a launch's logits in an array that it leaves at zero, and its two sets of
+    ready counters alternate from launch to launch: launches of different lengths (some of them two-kernel
+    launches of one or two tokens in between) must not see anything of each other, nor must a reset."""
+    wl = synth.QWEN.with_(L=20, S=200, d=512, C=15)
+    Wr = wl.router()
+    xs = np.stack(list(wl.hidden_trace(41)))
+    eng, o = mb.engine_for(wl, ffn_impl=mb.FFN_SIMT), H.oracle_for(wl)
+    eng.set_router(H.to_dev(Wr))
+    assert eng.router_kernel_kind(8) == mb.ROUTER_FUSED and eng.router_kernel_kind(2) == mb.ROUTER_RESIDENT_TAIL
+    near, dz = follow_chunked(eng, o, Wr, xs[:33], [8, 3, 1, 8, 5, 2, 6], None)
+    eng.reset()
+    o = H.oracle_for(wl)
+    near2, dz2 = follow_chunked(eng, o, Wr, xs[33:], [5, 3], mb.ROUTER_FUSED)
+    print("varying launches: %d near ties, max logit err %.2e" % (near + near2, max(dz, dz2)))
     eng.close()
 
 
