@@ -137,7 +137,7 @@ route_fused_kernel(const __grid_constant__ Maps maps, const FusedArgs args, cons
       const int t = i / a.n_tiles, tile = i % a.n_tiles;
       const size_t grow = (size_t)(t * a.L + l) * a.S + tile * kTileM + row;
       const bool row_ok = tile * kTileM + row < a.S;
-      if (!drain_pair<true>(a, m, tmem_base, kp, (uint32_t)i, quad, lane, args.Z + grow * a.E, row_ok, args.err, 35u)) break;
+      if (!drain_pair<true>(a, m, tmem_base, kp.n_k(i), (uint32_t)i, quad, lane, args.Z + grow * a.E, row_ok, args.err, 35u)) break;
       // Once per token (after its last stream tile; the tail consumes whole tokens): this warp's additions of the
       // token's pairs are ordered before its progress word for the other warps of the CTA.  The fence waits until
       // the reductions have been performed in L2, a round trip of 2-3 us here.

@@ -50,7 +50,7 @@ router_gemm_res_kernel(const __grid_constant__ Maps maps, const ResArgs args) {
     for (int i = g; i < n_pairs; i += args.TG, ++it) {
       const int t = i / a.n_tiles, tile = i % a.n_tiles;
       const int row0 = (t * a.L + l) * a.S + tile * kTileM;
-      if (!drain_pair<false>(a, m, tmem_base, kp, it, quad, lane, Zp + (size_t)(row0 + row) * a.E, tile * kTileM + row < a.S,
+      if (!drain_pair<false>(a, m, tmem_base, kp.n_k(i), it, quad, lane, Zp + (size_t)(row0 + row) * a.E, tile * kTileM + row < a.S,
                       args.err, 25u))
         break;
     }

@@ -91,14 +91,31 @@ __device__ __forceinline__ Smem carve(uint8_t* smem_raw, const Geometry& a) {
   return m;
 }
 
-// This CTA's K part: slabs [k_begin, k_begin + n_k).
+// This CTA's K part.  Every part owns slabs / KS slabs of its own, [k_begin, k_begin + n_own).  The slabs % KS
+// that are left over (the last ones) are shared: the parts form as many groups as there are left-over slabs, every
+// member of a group keeps the group's slab resident beside its own, and for the i-th (token, stream tile) pair of
+// the layer the member i mod gsize adds it to its reduction.  Over the pairs every part then does the same work
+// to within one slab per gsize pairs (with whole extra slabs per part, 32 slabs over 6 parts are 6,6,5,5,5,5 and
+// the parts with six set the pace of their layer).
 struct KPart {
-  int k_begin, n_k;
+  int k_begin, n_own;
+  int shared;          // the group's shared slab, or -1
+  int gsize, member;   // members of the group, this part's index among them
+  __device__ __forceinline__ int n_res() const { return n_own + (shared >= 0 ? 1 : 0); }        // resident slabs
+  __device__ __forceinline__ int n_k(int pair) const {                                           // slabs of a pair
+    return n_own + (shared >= 0 && pair % gsize == member ? 1 : 0);
+  }
+  __device__ __forceinline__ int slab(int j) const { return j < n_own ? k_begin + j : shared; }  // j-th of a pair
 };
 __device__ __forceinline__ KPart k_part_of(const Geometry& a, int ks) {
   const int k_base = a.slabs / a.KS, k_rem = a.slabs % a.KS;
   KPart p;
-  p.k_begin = ks * k_base + min(ks, k_rem), p.n_k = k_base + (ks < k_rem ? 1 : 0);
+  p.k_begin = ks * k_base, p.n_own = k_base, p.shared = -1, p.gsize = 1, p.member = 0;
+  if (k_rem > 0) {
+    const int g = ks * k_rem / a.KS;                                   // groups are runs of consecutive parts
+    const int first = (g * a.KS + k_rem - 1) / k_rem, next = ((g + 1) * a.KS + k_rem - 1) / k_rem;
+    p.shared = a.KS * k_base + g, p.gsize = next - first, p.member = ks - first;
+  }
   return p;
 }
 
@@ -124,11 +141,11 @@ __device__ __forceinline__ void produce(const Maps& maps, const Geometry& a, con
                                         int step, uint32_t* err, uint32_t code0) {
   const uint32_t term_bytes = (uint32_t)a.Epad * kRowBytes, slab_bytes = 3u * term_bytes;
   const int n_pairs = a.n_steps * a.n_tiles;
-  mbar_expect_tx(m.bar_res, (uint32_t)kp.n_k * slab_bytes);
-  for (int j = 0; j < kp.n_k; ++j)
+  mbar_expect_tx(m.bar_res, (uint32_t)kp.n_res() * slab_bytes);
+  for (int j = 0; j < kp.n_res(); ++j)
 #pragma unroll
     for (int q = 0; q < 3; ++q)
-      tma_load_3d(m.base + (uint32_t)j * slab_bytes + q * term_bytes, &maps.w, (kp.k_begin + j) * kTileK, 0,
+      tma_load_3d(m.base + (uint32_t)j * slab_bytes + q * term_bytes, &maps.w, kp.slab(j) * kTileK, 0,
                   q * a.L_terms + a.l0 + l, m.bar_res);
   uint32_t stage = 0, phase = 0;
   for (int i = first; i < n_pairs; i += step) {
@@ -136,11 +153,12 @@ __device__ __forceinline__ void produce(const Maps& maps, const Geometry& a, con
     const int row0 = (t * a.L + l) * a.S + tile * kTileM;
     // rows of the copy: a whole tile, or the ragged last tile of the layer rounded up to the box of maps.x
     const int n_box = (min(kTileM, a.S - tile * kTileM) + kXBox - 1) / kXBox;
-    for (int j = 0; j < kp.n_k; ++j) {
+    const int n_k = kp.n_k(i);
+    for (int j = 0; j < n_k; ++j) {
       if (!mbar_wait(m.bar_empty + 8 * stage, phase ^ 1u, m.abort_flag, err, code0)) return;
       const uint32_t sa = m.ring + stage * kStageBytes, full = m.bar_full + 8 * stage;
       mbar_expect_tx(full, (uint32_t)n_box * kXBox * kRowBytes);
-      tma_load_2d(sa, n_box == kTileM / kXBox ? &maps.xt : &maps.x, (kp.k_begin + j) * kTileK, row0, full);
+      tma_load_2d(sa, n_box == kTileM / kXBox ? &maps.xt : &maps.x, kp.slab(j) * kTileK, row0, full);
       if (++stage == (uint32_t)a.n_stages) stage = 0, phase ^= 1u;
     }
   }
@@ -159,7 +177,8 @@ __device__ __forceinline__ void issue_mmas(const Geometry& a, const Smem& m, uin
     const uint32_t buf = it & 1u, acc_phase = (it >> 1) & 1u;
     if (!mbar_wait(m.bar_tempty + 8 * buf, acc_phase ^ 1u, m.abort_flag, err, code0 + 2u)) return;
     tc_fence_after();
-    for (int j = 0; j < kp.n_k; ++j) {
+    const int n_k = kp.n_k(i);
+    for (int j = 0; j < n_k; ++j) {
       if (!mbar_wait(m.bar_full + 8 * stage, phase, m.abort_flag, err, code0 + 3u)) return;
       tc_fence_after();
       const uint32_t d_set = tmem_base + buf * kBufCols + (uint32_t)(j / kSetSlabs) * set_cols;
@@ -183,16 +202,17 @@ __device__ __forceinline__ void red_add4(float* q, float a, float b, float c, fl
 // partial logits of rows row0 + quad*32 + lane (zrow: the row in the part's [rows][E] array); then releases the
 // TMEM buffer.  With ADD the partial logits are added to zrow instead (fp32 reductions performed in L2; the K
 // parts of a layer then share one array that starts at zero, and the order of the additions is that of arrival).
-// Returns false if the CTA is giving up.  it = how many pairs this CTA has finished before.
+// Returns false if the CTA is giving up.  it = how many pairs this CTA has finished before; n_k = slabs that
+// went into this pair.
 template <bool ADD>
-__device__ __forceinline__ bool drain_pair(const Geometry& a, const Smem& m, uint32_t tmem_base, KPart kp, uint32_t it,
+__device__ __forceinline__ bool drain_pair(const Geometry& a, const Smem& m, uint32_t tmem_base, int n_k, uint32_t it,
                                            int quad, int lane, float* zrow, bool row_ok, uint32_t* err, uint32_t code) {
   const uint32_t buf = it & 1u, acc_phase = (it >> 1) & 1u;
   if (!mbar_wait(m.bar_tfull + 8 * buf, acc_phase, m.abort_flag, err, code)) return false;
   tc_fence_after();
   const uint32_t set_cols = 3u * (uint32_t)a.Epad;
   const uint32_t t0 = tmem_base + ((uint32_t)(quad * 32) << 16) + buf * kBufCols;
-  const int n_sets = (kp.n_k + kSetSlabs - 1) / kSetSlabs;
+  const int n_sets = (n_k + kSetSlabs - 1) / kSetSlabs;
   const bool vec4 = (a.E & 3) == 0;
   for (int c = 0; c < a.Epad; c += 16) {
     float acc[16];
