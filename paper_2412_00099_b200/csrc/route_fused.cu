@@ -195,7 +195,8 @@ route_fused_kernel(const __grid_constant__ Maps maps, const FusedArgs args, cons
 }
 
 int group_of(int E) { return E <= 8 ? 1 : E <= 16 ? 2 : E <= 32 ? 4 : 8; }
-int tail_bucket(int tail_warps) { return tail_warps <= 8 ? 8 : tail_warps <= 12 ? 12 : 16; }
+// (13 tail warps are the most that leave a thread 96 registers: 7 + 13 = 20 warps, five per scheduler)
+int tail_bucket(int tail_warps) { return tail_warps <= 8 ? 8 : tail_warps <= 13 ? 13 : 16; }
 
 template <int G, int KMAX, int TW>
 cudaError_t launch_one(const Maps& m, const FusedArgs& a, const RouteParams& p, cudaStream_t st) {
@@ -230,10 +231,10 @@ int resident_ctas() {
 
 // The instantiations: group size by expert count, selections per token, tail warps.
 #define MCCE_FUSED_FOR_EACH(X)                                                                             \
-  X(1, 4, 8) X(1, 8, 8) X(1, 4, 12) X(1, 8, 12) X(1, 4, 16) X(1, 8, 16)                                      \
-  X(2, 4, 8) X(2, 8, 8) X(2, 16, 8) X(2, 4, 12) X(2, 8, 12) X(2, 16, 12) X(2, 4, 16) X(2, 8, 16) X(2, 16, 16) \
-  X(4, 4, 8) X(4, 8, 8) X(4, 16, 8) X(4, 4, 12) X(4, 8, 12) X(4, 16, 12) X(4, 4, 16) X(4, 8, 16) X(4, 16, 16) \
-  X(8, 4, 8) X(8, 8, 8) X(8, 16, 8) X(8, 4, 12) X(8, 8, 12) X(8, 16, 12) X(8, 4, 16) X(8, 8, 16) X(8, 16, 16)
+  X(1, 4, 8) X(1, 8, 8) X(1, 4, 13) X(1, 8, 13) X(1, 4, 16) X(1, 8, 16)                                      \
+  X(2, 4, 8) X(2, 8, 8) X(2, 16, 8) X(2, 4, 13) X(2, 8, 13) X(2, 16, 13) X(2, 4, 16) X(2, 8, 16) X(2, 16, 16) \
+  X(4, 4, 8) X(4, 8, 8) X(4, 16, 8) X(4, 4, 13) X(4, 8, 13) X(4, 16, 13) X(4, 4, 16) X(4, 8, 16) X(4, 16, 16) \
+  X(8, 4, 8) X(8, 8, 8) X(8, 16, 8) X(8, 4, 13) X(8, 8, 13) X(8, 16, 13) X(8, 4, 16) X(8, 8, 16) X(8, 16, 16)
 
 int k_bucket(int K) { return K <= 4 ? 4 : K <= 8 ? 8 : 16; }
 
