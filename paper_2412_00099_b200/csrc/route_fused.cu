@@ -6,10 +6,11 @@
 // A layer belongs to KS CTAs (one K part of the reduction each).  Warps 0-5 of a CTA are the GEMM (TMA
 // producer, MMA issuer, four epilogue warps).  An epilogue warp adds the partial logits of its K part for its
 // 32 rows of the (token, stream tile) into the launch's logits array (fp32 reductions in L2; the array is zero
-// at launch) and notes its progress in shared memory.  Warp 6 publishes: once all four epilogue warps are
-// through with a pair it issues the device-wide fence and adds the CTA's four counts to the pair's counter.  (A
-// fence takes about 3 us while the device streams hidden states; issued by the epilogue warps themselves it
-// made them, not the tensor core, set the pace: 4.8 us per tile instead of 2.7.)  The remaining warps are the
+// at launch) and, after the last stream tile of a token, notes its progress in shared memory.  Warp 6 publishes:
+// once all four epilogue warps are through with a token it issues the device-wide fence and adds the CTA's four
+// counts to the counters of the token's pairs.  (A fence takes about 3 us while the device streams hidden
+// states; issued by the epilogue warps themselves, tile by tile, it made them, not the tensor core, set the pace:
+// 4.8 us per tile instead of 2.7.)  The remaining warps are the
 // tail: the S streams of the layer are dealt out to its KS CTAs, a group of lanes per stream as in
 // route_group.cuh.  Before a token they wait (bounded) until all KS CTAs of the layer have counted in on the
 // tiles they read, then read the sums (L2-coherent loads) and put the zeros back.  The launch is cooperative, so
